@@ -88,6 +88,18 @@ const char* jupiter_last_cuda_error(const jupiter_ctx* ctx);
  * JUPITER_ERR_CUDA if the stream reports an error, else JUPITER_OK. */
 jupiter_status jupiter_poll_device_status(jupiter_ctx* ctx, void* stream);
 
+/* Failure-detection aid; the paper has no counterpart.  Every device-side wait of the tensor-core kernels
+ * (on a TMA copy, on a tensor-core result) is bounded: when its limit of SM clocks runs out the kernel sets the
+ * ctx status word, waits for its own copies in flight, frees its tensor memory and returns normally.  From then on
+ * and until jupiter_poll_device_status has reported JUPITER_ERR_TIMEOUT (which clears the word), kernels of this
+ * ctx that have to wait give up as well, and the outputs of those launches are undefined.
+ * This call enqueues one tiny kernel whose single wait is on a barrier that nobody arrives at, with a limit of
+ * `limit_cycles` SM clocks (1 .. 2e9; JUPITER_ERR_INVALID_ARG otherwise): the wait runs out, the status word
+ * is set and the kernel returns -- nothing faults, the context and the GPU stay usable.  It lets a caller (and
+ * the tests) exercise the reporting path: the next jupiter_poll_device_status returns JUPITER_ERR_TIMEOUT once,
+ * later polls JUPITER_OK, and later calls compute as usual. */
+jupiter_status jupiter_wait_probe(jupiter_ctx* ctx, int64_t limit_cycles, void* stream);
+
 /* Number of this library's kernel launches enqueued through the ctx so far. */
 uint64_t jupiter_launch_count(const jupiter_ctx* ctx);
 
@@ -191,6 +203,21 @@ jupiter_status jupiter_branch_append_attn(jupiter_ctx* ctx, const void* q, const
                                           const jupiter_kv_cache* suffix, const int32_t* d_suffix_len,
                                           int32_t max_suffix_len, int32_t n_branches, int32_t q_heads,
                                           int32_t q_len, float scale, float* out, float* lse, void* stream);
+
+/* Tuning and testing aid; the paper has no counterpart.  The branch calls (jupiter_branch_attn, _tree,
+ * jupiter_branch_append_attn) pick one of three kernels from the shape: a streaming kernel for few stacked
+ * query rows per kv head (decode), a tensor-core kernel (tcgen05 / TMEM) for many rows with head_dim 128, and a
+ * general split-KV kernel.  This call pins the choice for later calls on `ctx`; JUPITER_BRANCH_AUTO restores the
+ * default.  A call whose shape the pinned kernel cannot take returns JUPITER_ERR_UNSUPPORTED (the tensor-core
+ * kernel needs head_dim 128, scale > 0, a group size q_heads / kv_heads that is a power of two, and
+ * q_len * group >= 5).  All three give the same result up to rounding. */
+typedef enum {
+  JUPITER_BRANCH_AUTO = 0,
+  JUPITER_BRANCH_STREAM = 1,
+  JUPITER_BRANCH_SPLIT_KV = 2,
+  JUPITER_BRANCH_TENSOR_CORE = 3
+} jupiter_branch_kernel;
+jupiter_status jupiter_select_branch_kernel(jupiter_ctx* ctx, jupiter_branch_kernel which);
 
 /* Prefill of a branch's own prompt against the shared prefix (Sec. V-B: every point-extending
  * request first ingests its own instruction while sharing the prompt KVCache).  Chunked-prefill

@@ -6,8 +6,10 @@ newer); there is no other implementation behind these names.
 """
 from .binding import (branch_attn_noalloc, plan_sequence_partition, Context, JupiterError, cache_desc, jupiter_kv_cache, lib, library_path, EXPORTS,
                       STATUS_NAMES, OK, ERR_INVALID_ARG, ERR_OUT_OF_RANGE, ERR_UNSUPPORTED, ERR_ALIGNMENT,
-                      ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT)
+                      ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT, BRANCH_AUTO, BRANCH_STREAM, BRANCH_SPLIT_KV,
+                      BRANCH_TENSOR_CORE)
 
 __all__ = ["branch_attn_noalloc", "plan_sequence_partition", "Context", "JupiterError", "cache_desc", "jupiter_kv_cache", "lib", "library_path", "EXPORTS",
            "STATUS_NAMES", "OK", "ERR_INVALID_ARG", "ERR_OUT_OF_RANGE", "ERR_UNSUPPORTED", "ERR_ALIGNMENT",
-           "ERR_WORKSPACE", "ERR_CUDA", "ERR_TIMEOUT"]
+           "ERR_WORKSPACE", "ERR_CUDA", "ERR_TIMEOUT", "BRANCH_AUTO", "BRANCH_STREAM", "BRANCH_SPLIT_KV",
+           "BRANCH_TENSOR_CORE"]

@@ -22,6 +22,7 @@ STATUS_NAMES = {
     0: "JUPITER_OK", 1: "JUPITER_ERR_INVALID_ARG", 2: "JUPITER_ERR_OUT_OF_RANGE", 3: "JUPITER_ERR_UNSUPPORTED",
     4: "JUPITER_ERR_ALIGNMENT", 5: "JUPITER_ERR_WORKSPACE", 6: "JUPITER_ERR_CUDA", 7: "JUPITER_ERR_TIMEOUT",
 }
+BRANCH_AUTO, BRANCH_STREAM, BRANCH_SPLIT_KV, BRANCH_TENSOR_CORE = range(4)
 (OK, ERR_INVALID_ARG, ERR_OUT_OF_RANGE, ERR_UNSUPPORTED, ERR_ALIGNMENT, ERR_WORKSPACE, ERR_CUDA,
  ERR_TIMEOUT) = range(8)
 
@@ -31,7 +32,7 @@ EXPORTS = (
     "jupiter_chunk_prefill_attn", "jupiter_branch_attn", "jupiter_branch_attn_noalloc",
     "jupiter_plan_sequence_partition", "jupiter_branch_attn_tree", "jupiter_branch_prefill_attn",
     "jupiter_chunk_prefill_append_attn", "jupiter_branch_append_attn", "jupiter_read_probe",
-    "jupiter_kv_compact",
+    "jupiter_kv_compact", "jupiter_wait_probe", "jupiter_select_branch_kernel",
 )
 
 
@@ -71,6 +72,10 @@ def _load() -> ctypes.CDLL:
     lib.jupiter_launch_count.restype = ctypes.c_uint64
     lib.jupiter_kv_compact.argtypes = [c_void_p, P(jupiter_kv_cache), c_int32, c_void_p, c_void_p, c_void_p, c_void_p]
     lib.jupiter_kv_compact.restype = ctypes.c_int
+    lib.jupiter_select_branch_kernel.argtypes = [c_void_p, ctypes.c_int]
+    lib.jupiter_select_branch_kernel.restype = ctypes.c_int
+    lib.jupiter_wait_probe.argtypes = [c_void_p, c_int64, c_void_p]
+    lib.jupiter_wait_probe.restype = ctypes.c_int
     lib.jupiter_read_probe.argtypes = [c_void_p, c_void_p, c_size_t, c_void_p, c_void_p]
     lib.jupiter_read_probe.restype = ctypes.c_int
     lib.jupiter_kv_append.argtypes = [c_void_p, P(jupiter_kv_cache), c_void_p, c_void_p, c_int32, c_int32,
@@ -163,6 +168,12 @@ class Context:
 
     def read_probe(self, src, nbytes: int, out, stream=None):
         self._check(lib.jupiter_read_probe(self._h, _ptr(src), nbytes, _ptr(out), _stream(stream)))
+
+    def select_branch_kernel(self, which: int):
+        self._check(lib.jupiter_select_branch_kernel(self._h, int(which)))
+
+    def wait_probe(self, limit_cycles: int, stream=None):
+        self._check(lib.jupiter_wait_probe(self._h, int(limit_cycles), _stream(stream)))
 
     def poll_device_status(self, stream=None) -> int:
         return int(lib.jupiter_poll_device_status(self._h, _stream(stream)))

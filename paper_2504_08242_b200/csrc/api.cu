@@ -5,6 +5,7 @@
 #include <new>
 
 #include "../../include/jupiter.h"
+#include "host_checks.h"
 #include "kernels.h"
 
 struct jupiter_ctx {
@@ -13,40 +14,22 @@ struct jupiter_ctx {
   void* workspace;
   size_t workspace_bytes;
   int* d_status;
+  long long wait_limit;  // SM clocks a device-side wait may last
+  int branch_kernel;     // jupiter_branch_kernel: which kernel the branch calls use
   uint64_t launches;
   char err[256];
 };
 
 namespace {
 
+using jup::aligned16;
 using jup::bf16;
 using jup::CacheView;
-
-inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+using jup::check_cache;
 
 jupiter_status cuda_fail(jupiter_ctx* ctx, cudaError_t e, const char* where) {
   if (ctx) std::snprintf(ctx->err, sizeof ctx->err, "%s: %s", where, cudaGetErrorString(e));
   return JUPITER_ERR_CUDA;
-}
-
-// Validates a cache descriptor and turns it into a CacheView.
-jupiter_status check_cache(const jupiter_kv_cache* c, CacheView* out) {
-  if (!c || !c->k || !c->v) return JUPITER_ERR_INVALID_ARG;
-  if (c->batch <= 0 || c->kv_heads <= 0 || c->capacity <= 0) return JUPITER_ERR_INVALID_ARG;
-  if (c->head_dim != 64 && c->head_dim != 128) return JUPITER_ERR_UNSUPPORTED;
-  if (c->stride_row < c->head_dim || c->stride_head < 0 || c->stride_batch < 0) return JUPITER_ERR_INVALID_ARG;
-  if (!aligned16(c->k) || !aligned16(c->v)) return JUPITER_ERR_ALIGNMENT;
-  if ((c->stride_row % 8) || (c->stride_head % 8) || (c->stride_batch % 8)) return JUPITER_ERR_ALIGNMENT;
-  out->k = static_cast<const bf16*>(c->k);
-  out->v = static_cast<const bf16*>(c->v);
-  out->batch = c->batch;
-  out->kv_heads = c->kv_heads;
-  out->capacity = c->capacity;
-  out->head_dim = c->head_dim;
-  out->sb = c->stride_batch;
-  out->sh = c->stride_head;
-  out->sr = c->stride_row;
-  return JUPITER_OK;
 }
 
 struct DeviceGuard {
@@ -93,6 +76,7 @@ jupiter_status jupiter_create(jupiter_ctx** out_ctx, int device, size_t workspac
   ctx->device = device;
   ctx->sm_count = prop.multiProcessorCount;
   ctx->workspace_bytes = workspace_bytes ? workspace_bytes : (size_t(64) << 20);
+  ctx->wait_limit = 2000000000ll;
   DeviceGuard guard(device);
   e = cudaMalloc(&ctx->workspace, ctx->workspace_bytes);
   if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&ctx->d_status), 256);
@@ -138,6 +122,21 @@ jupiter_status jupiter_poll_device_status(jupiter_ctx* ctx, void* stream) {
     return JUPITER_ERR_TIMEOUT;
   }
   return JUPITER_OK;
+}
+
+jupiter_status jupiter_select_branch_kernel(jupiter_ctx* ctx, jupiter_branch_kernel which) {
+  if (!ctx || which < JUPITER_BRANCH_AUTO || which > JUPITER_BRANCH_TENSOR_CORE) return JUPITER_ERR_INVALID_ARG;
+  ctx->branch_kernel = which;
+  return JUPITER_OK;
+}
+
+jupiter_status jupiter_wait_probe(jupiter_ctx* ctx, int64_t limit_cycles, void* stream) {
+  if (!ctx || limit_cycles <= 0 || limit_cycles > 2000000000ll) return JUPITER_ERR_INVALID_ARG;
+  DeviceGuard guard(ctx->device);
+  jup::LaunchInfo li{ctx->sm_count, 0};
+  cudaError_t e = jup::launch_wait_probe(ctx->d_status, limit_cycles, static_cast<cudaStream_t>(stream), li);
+  ctx->launches += li.launches;
+  return e == cudaSuccess ? JUPITER_OK : cuda_fail(ctx, e, "wait_probe");
 }
 
 jupiter_status jupiter_read_probe(jupiter_ctx* ctx, const void* src, size_t bytes, uint32_t* out, void* stream) {
@@ -200,7 +199,7 @@ jupiter_status jupiter_chunk_prefill_attn(jupiter_ctx* ctx, const void* q, const
   jupiter_status s = check_cache(cache, &c);
   if (s != JUPITER_OK) return s;
   if (q_heads <= 0 || q_len <= 0 || q_heads % c.kv_heads != 0) return JUPITER_ERR_INVALID_ARG;
-  if (!(scale == scale)) return JUPITER_ERR_INVALID_ARG;
+  if (!jup::scale_ok(scale)) return JUPITER_ERR_INVALID_ARG;
   if (pos < 0 || static_cast<int64_t>(pos) + q_len > c.capacity) return JUPITER_ERR_OUT_OF_RANGE;
   if (!aligned16(q) || !aligned16(out)) return JUPITER_ERR_ALIGNMENT;
   DeviceGuard guard(ctx->device);
@@ -224,7 +223,7 @@ jupiter_status jupiter_chunk_prefill_append_attn(jupiter_ctx* ctx, const void* q
   jupiter_status s = check_cache(cache, &c);
   if (s != JUPITER_OK) return s;
   if (q_heads <= 0 || q_len <= 0 || q_heads % c.kv_heads != 0) return JUPITER_ERR_INVALID_ARG;
-  if (!(scale == scale)) return JUPITER_ERR_INVALID_ARG;
+  if (!jup::scale_ok(scale)) return JUPITER_ERR_INVALID_ARG;
   if (pos < 0 || static_cast<int64_t>(pos) + q_len > c.capacity) return JUPITER_ERR_OUT_OF_RANGE;
   if (!aligned16(q) || !aligned16(out) || !aligned16(k_new) || !aligned16(v_new)) return JUPITER_ERR_ALIGNMENT;
   DeviceGuard guard(ctx->device);
@@ -262,7 +261,7 @@ jupiter_status jupiter_branch_prefill_attn(jupiter_ctx* ctx, const void* q, cons
     if (prefix_len > pfx.capacity) return JUPITER_ERR_OUT_OF_RANGE;
   }
   if (q_heads <= 0 || q_len <= 0 || q_heads % c.kv_heads != 0) return JUPITER_ERR_INVALID_ARG;
-  if (!(scale == scale)) return JUPITER_ERR_INVALID_ARG;
+  if (!jup::scale_ok(scale)) return JUPITER_ERR_INVALID_ARG;
   if (pos < 0 || static_cast<int64_t>(pos) + q_len > c.capacity) return JUPITER_ERR_OUT_OF_RANGE;
   if (!aligned16(q) || !aligned16(out)) return JUPITER_ERR_ALIGNMENT;
   if (!jup::prefill_tc_supported(c, scale)) return JUPITER_ERR_UNSUPPORTED;  // head_dim 128 and scale > 0 only
@@ -297,20 +296,43 @@ static jupiter_status branch_attn_impl(jupiter_ctx* ctx, const void* q, const ju
   if (n_branches <= 0 || n_branches != sfx.batch) return JUPITER_ERR_INVALID_ARG;
   if (q_heads <= 0 || q_heads % sfx.kv_heads != 0 || q_len <= 0) return JUPITER_ERR_INVALID_ARG;
   if (q_len > 16) return JUPITER_ERR_UNSUPPORTED;
-  if (!(scale == scale)) return JUPITER_ERR_INVALID_ARG;
+  if (!jup::scale_ok(scale)) return JUPITER_ERR_INVALID_ARG;
   if (max_suffix_len < q_len || max_suffix_len > sfx.capacity) return JUPITER_ERR_OUT_OF_RANGE;
   if (!aligned16(q) || !aligned16(out)) return JUPITER_ERR_ALIGNMENT;
-  const size_t need = jup::branch_workspace_bytes(prefix_len, max_suffix_len, n_branches, q_heads, sfx.kv_heads, q_len,
-                                                  sfx.head_dim, ctx->sm_count);
-  if (need > ctx->workspace_bytes) return JUPITER_ERR_WORKSPACE;
+  // which kernel: few stacked rows per kv head stream through clusters (no scratch); many rows with head_dim 128 go
+  // to the tensor-core kernel (which adapts to the scratch it is given); the rest to the split-KV kernel, the only
+  // one that can find the scratch too small
+  const bool tc_ok = jup::branch_tc_supported(sfx, prefix_len, max_suffix_len, n_branches, q_heads, q_len, scale,
+                                              ctx->sm_count);
+  bool use_stream, use_tc;
+  switch (ctx->branch_kernel) {
+    case JUPITER_BRANCH_STREAM: use_stream = true, use_tc = false; break;
+    case JUPITER_BRANCH_SPLIT_KV: use_stream = use_tc = false; break;
+    case JUPITER_BRANCH_TENSOR_CORE:
+      if (!tc_ok) return JUPITER_ERR_UNSUPPORTED;
+      use_stream = false, use_tc = true;
+      break;
+    default:
+      use_stream = jup::branch_stream_preferred(n_branches, q_heads, sfx.kv_heads, q_len, ctx->sm_count);
+      use_tc = !use_stream && tc_ok;
+  }
+  if (!use_stream && !use_tc &&
+      jup::branch_workspace_bytes(prefix_len, max_suffix_len, n_branches, q_heads, sfx.kv_heads, q_len, sfx.head_dim,
+                                  ctx->sm_count) > ctx->workspace_bytes)
+    return JUPITER_ERR_WORKSPACE;
   DeviceGuard guard(ctx->device);
   jup::LaunchInfo li{ctx->sm_count, 0};
   cudaError_t e;
-  if (jup::branch_stream_preferred(n_branches, q_heads, sfx.kv_heads, q_len, ctx->sm_count))
+  if (use_stream)
     e = jup::launch_branch_stream(static_cast<const bf16*>(q), pfx, prefix_len, sfx, d_suffix_len, d_tree_mask,
                                   max_suffix_len, n_branches, q_heads, q_len, scale, out, lse,
                                   static_cast<cudaStream_t>(stream), li, static_cast<const bf16*>(k_new),
                                   static_cast<const bf16*>(v_new));
+  else if (use_tc)
+    e = jup::launch_branch_tc(static_cast<const bf16*>(q), pfx, prefix_len, sfx, d_suffix_len, d_tree_mask,
+                              max_suffix_len, n_branches, q_heads, q_len, scale, out, lse, ctx->d_status,
+                              ctx->wait_limit, ctx->workspace, ctx->workspace_bytes, static_cast<cudaStream_t>(stream),
+                              li, static_cast<const bf16*>(k_new), static_cast<const bf16*>(v_new));
   else
     e = jup::launch_branch(static_cast<const bf16*>(q), pfx, prefix_len, sfx, d_suffix_len, d_tree_mask,
                            max_suffix_len, n_branches, q_heads, q_len, scale, out, lse, ctx->workspace,

@@ -20,6 +20,7 @@
 // Scratch layout: [64 KiB of int32 counters, one per (branch, kv head), zero between calls]
 // [O partials][(m, l) partials].  The merging CTA puts each counter back to zero.
 #include "attn_keysplit.cuh"
+#include "host_checks.h"
 #include "kernels.h"
 
 namespace jup {
@@ -363,8 +364,8 @@ __global__ void __launch_bounds__(128) branch_merge_kernel(BranchParams p) {
 template <int D, int MT, int STAGES, bool FUSED_MERGE>
 static cudaError_t launch_branch_d(const BranchParams& p, cudaStream_t st, LaunchInfo& li) {
   constexpr int smem = KeySplitCfg<D, MT, STAGES>::SMEM_BYTES;
-  static bool attr_done = false;
-  if (!attr_done) {
+  static PerDeviceOnce attr_done;
+  if (!attr_done.done()) {
     cudaError_t e = cudaFuncSetAttribute(branch_attn_kernel<D, MT, STAGES, FUSED_MERGE>,
                                          cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e == cudaSuccess)
@@ -374,7 +375,7 @@ static cudaError_t launch_branch_d(const BranchParams& p, cudaStream_t st, Launc
       e = cudaFuncSetAttribute(branch_merge_kernel<D>, cudaFuncAttributePreferredSharedMemoryCarveout,
                                cudaSharedmemCarveoutMaxShared);
     if (e != cudaSuccess) return e;
-    attr_done = true;
+    attr_done.set();
   }
   const unsigned grid = static_cast<unsigned>(p.pl.items_p + p.pl.items_s);
   cudaError_t e = launch_pdl(branch_attn_kernel<D, MT, STAGES, FUSED_MERGE>, dim3(grid), dim3(128), smem, st, p);

@@ -9,6 +9,7 @@
 #include <mutex>
 
 #include "../../include/jupiter.h"
+#include "host_checks.h"
 #include "kernels.h"
 
 // The scratch itself: part of the loaded module, so every GPU that loads the library
@@ -25,27 +26,6 @@ struct PerDevice {
 };
 PerDevice g_dev[kMaxDevices];
 std::mutex g_mu;
-
-inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
-
-jupiter_status view_of(const jupiter_kv_cache* c, jup::CacheView* out) {
-  if (!c || !c->k || !c->v) return JUPITER_ERR_INVALID_ARG;
-  if (c->batch <= 0 || c->kv_heads <= 0 || c->capacity <= 0) return JUPITER_ERR_INVALID_ARG;
-  if (c->head_dim != 64 && c->head_dim != 128) return JUPITER_ERR_UNSUPPORTED;
-  if (c->stride_row < c->head_dim || c->stride_head < 0 || c->stride_batch < 0) return JUPITER_ERR_INVALID_ARG;
-  if (!aligned16(c->k) || !aligned16(c->v)) return JUPITER_ERR_ALIGNMENT;
-  if ((c->stride_row % 8) || (c->stride_head % 8) || (c->stride_batch % 8)) return JUPITER_ERR_ALIGNMENT;
-  out->k = static_cast<const jup::bf16*>(c->k);
-  out->v = static_cast<const jup::bf16*>(c->v);
-  out->batch = c->batch;
-  out->kv_heads = c->kv_heads;
-  out->capacity = c->capacity;
-  out->head_dim = c->head_dim;
-  out->sb = c->stride_batch;
-  out->sh = c->stride_head;
-  out->sr = c->stride_row;
-  return JUPITER_OK;
-}
 
 // One-time set-up for the current device.  In host code the name g_noalloc_scratch is only
 // a host-side handle of the symbol, not something a kernel can dereference; the address
@@ -78,12 +58,12 @@ extern "C" jupiter_status jupiter_branch_attn_noalloc(const void* q, const jupit
                                                       float scale, float* out, float* lse, void* stream) {
   if (!q || !out || !d_suffix_len) return JUPITER_ERR_INVALID_ARG;
   jup::CacheView sfx;
-  jupiter_status s = view_of(suffix, &sfx);
+  jupiter_status s = jup::check_cache(suffix, &sfx);
   if (s != JUPITER_OK) return s;
   jup::CacheView pfx = sfx;
   if (prefix_len < 0) return JUPITER_ERR_INVALID_ARG;
   if (prefix_len > 0) {
-    s = view_of(prefix, &pfx);
+    s = jup::check_cache(prefix, &pfx);
     if (s != JUPITER_OK) return s;
     if (pfx.batch != 1 || pfx.kv_heads != sfx.kv_heads || pfx.head_dim != sfx.head_dim) return JUPITER_ERR_INVALID_ARG;
     if (prefix_len > pfx.capacity) return JUPITER_ERR_OUT_OF_RANGE;
@@ -91,9 +71,9 @@ extern "C" jupiter_status jupiter_branch_attn_noalloc(const void* q, const jupit
   if (n_branches <= 0 || n_branches != sfx.batch) return JUPITER_ERR_INVALID_ARG;
   if (q_heads <= 0 || q_heads % sfx.kv_heads != 0 || q_len <= 0) return JUPITER_ERR_INVALID_ARG;
   if (q_len > 16) return JUPITER_ERR_UNSUPPORTED;
-  if (!(scale == scale)) return JUPITER_ERR_INVALID_ARG;
+  if (!jup::scale_ok(scale)) return JUPITER_ERR_INVALID_ARG;
   if (max_suffix_len < q_len || max_suffix_len > sfx.capacity) return JUPITER_ERR_OUT_OF_RANGE;
-  if (!aligned16(q) || !aligned16(out)) return JUPITER_ERR_ALIGNMENT;
+  if (!jup::aligned16(q) || !jup::aligned16(out)) return JUPITER_ERR_ALIGNMENT;
 
   int dev = -1;
   if (cudaGetDevice(&dev) != cudaSuccess) return JUPITER_ERR_CUDA;

@@ -24,6 +24,7 @@
 // Fused KVCache write: with k_new / v_new the rows of this step's block are read from there
 // (they are not in the cache yet) and the warp that fetched them stores them into the suffix
 // rows [L_b - q_len, L_b) from shared memory.
+#include "host_checks.h"
 #include "kernels.h"
 #include "tc_common.cuh"
 
@@ -63,13 +64,7 @@ struct StreamCfg {
 };
 
 // Launch shape: warps per CTA, ring slots per warp, CTAs that fit one SM with that much shared memory.
-#ifndef JUP_STREAM_WARPS
-#define JUP_STREAM_WARPS 8
-#define JUP_STREAM_STAGES 2
-#define JUP_STREAM_CTAS_PER_SM 1
-#endif
-constexpr int kStreamWarps = JUP_STREAM_WARPS, kStreamStages = JUP_STREAM_STAGES,
-              kStreamCtasPerSm = JUP_STREAM_CTAS_PER_SM;
+constexpr int kStreamWarps = 8, kStreamStages = 2, kStreamCtasPerSm = 1;
 
 __device__ __forceinline__ void st_cluster_f4(uint32_t addr, float4 v) {
   asm volatile("st.shared::cluster.v4.f32 [%0], {%1, %2, %3, %4};\n" ::"r"(addr), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w)
@@ -479,15 +474,15 @@ __global__ void __launch_bounds__(NW * 32, kStreamCtasPerSm) branch_stream_kerne
 template <int D, int NW, int ST>
 static cudaError_t launch_stream_d(const StreamParams& p, int units, cudaStream_t st, LaunchInfo& li) {
   using Cfg = StreamCfg<D, NW, ST>;
-  static bool attr_done = false;
-  if (!attr_done) {
+  static PerDeviceOnce attr_done;
+  if (!attr_done.done()) {
     cudaError_t e = cudaFuncSetAttribute(branch_stream_kernel<D, NW, ST>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          Cfg::SMEM_BYTES);
     if (e == cudaSuccess)
       e = cudaFuncSetAttribute(branch_stream_kernel<D, NW, ST>, cudaFuncAttributePreferredSharedMemoryCarveout,
                                cudaSharedmemCarveoutMaxShared);
     if (e != cudaSuccess) return e;
-    attr_done = true;
+    attr_done.set();
   }
   li.launches += 1;
   return launch_pdl_cluster(branch_stream_kernel<D, NW, ST>, dim3(static_cast<unsigned>(units * p.cluster)),

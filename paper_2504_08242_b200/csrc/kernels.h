@@ -98,6 +98,22 @@ cudaError_t launch_branch_stream(const bf16* q, const CacheView& prefix, int pre
                                  cudaStream_t st, LaunchInfo& li, const bf16* k_new = nullptr,
                                  const bf16* v_new = nullptr);
 
+// Branch attention on tcgen05 / TMEM for many stacked rows per kv head (head_dim 128, positive finite scale, group
+// size a power of two): units of (kv head, 128 stacked rows) walk prefix + suffixes with one softmax state per row;
+// the CTAs that share a unit merge their partials through the scratch (last arriver, fixed order).  With too little
+// scratch the units are split over fewer CTAs, so the call never fails for lack of it.
+bool branch_tc_supported(const CacheView& suffix, int prefix_len, int max_suffix_len, int n_branches, int q_heads,
+                         int q_len, float scale, int sm_count);
+cudaError_t launch_branch_tc(const bf16* q, const CacheView& prefix, int prefix_len, const CacheView& suffix,
+                             const int32_t* d_suffix_len, const uint32_t* d_tree_mask, int max_suffix_len,
+                             int n_branches, int q_heads, int q_len, float scale, float* out, float* lse, int* status,
+                             long long wait_limit, void* workspace, size_t workspace_bytes, cudaStream_t st,
+                             LaunchInfo& li, const bf16* k_new = nullptr, const bf16* v_new = nullptr);
+
+// One CTA that waits, for at most limit_cycles SM clocks, on a barrier nobody arrives at, then reports through the
+// status word like any kernel whose bounded wait ran out.
+cudaError_t launch_wait_probe(int* status, long long limit_cycles, cudaStream_t st, LaunchInfo& li);
+
 // Moves the accepted rows of every sequence's draft block (q_len <= 16 rows at d_pos[b]) to the front of the block.
 cudaError_t launch_kv_compact(const CacheView& c, int q_len, const int32_t* d_pos, const int32_t* d_accept,
                               const int32_t* d_n_accept, cudaStream_t st, LaunchInfo& li);

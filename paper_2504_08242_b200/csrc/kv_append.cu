@@ -1,6 +1,7 @@
 // KVCache write (paper Sec. II-A; Sec. V-A step 3): token-major new K/V rows are
 // moved bit-exactly into head-major cache rows [pos_b, pos_b + n).  Pure data
 // movement, HBM-bound: every thread moves 16-byte chunks with 128-bit loads/stores.
+#include "host_checks.h"
 #include "kernels.h"
 
 namespace jup {
@@ -28,7 +29,7 @@ __global__ void __launch_bounds__(256) kv_append_kernel(AppendParams p) {
     const int t = static_cast<int>(r % p.n_rows);
     const int b = static_cast<int>(r / p.n_rows);
     const int pos = p.d_pos ? p.d_pos[b] : p.pos;
-    if (pos < 0 || pos + p.n_rows > p.capacity) continue;  // never form an address outside the cache
+    if (pos < 0 || pos > p.capacity - p.n_rows) continue;  // never form an address outside the cache (no overflow: n_rows <= capacity)
     const int64_t dst = b * p.sb + h * p.sh + static_cast<int64_t>(pos + t) * p.sr + c * 8;
     const uint4 kk = p.k_new[idx];
     const uint4 vv = p.v_new[idx];
@@ -62,12 +63,12 @@ cudaError_t launch_kv_append(const CacheView& c, const bf16* k_new, const bf16* 
   if (blocks > cap) blocks = cap;
   // Keep the SM's shared-memory carve-out where the attention kernels (which follow every append)
   // need it: a launch that prefers a different L1/shared split makes the SMs reconfigure in between.
-  static bool attr_done = false;
-  if (!attr_done) {
+  static PerDeviceOnce attr_done;
+  if (!attr_done.done()) {
     cudaError_t e = cudaFuncSetAttribute(kv_append_kernel, cudaFuncAttributePreferredSharedMemoryCarveout,
                                          cudaSharedmemCarveoutMaxShared);
     if (e != cudaSuccess) return e;
-    attr_done = true;
+    attr_done.set();
   }
   li.launches += 1;
   return launch_pdl(kv_append_kernel, dim3(static_cast<unsigned>(blocks)), dim3(threads), 0, st, p);

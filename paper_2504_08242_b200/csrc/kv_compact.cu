@@ -5,6 +5,7 @@
 //     row (pos_b + j)  <-  row (pos_b + accept[b][j])      j < n_accept[b], K and V, every kv head.
 // One CTA per (sequence, kv head): the accepted rows are staged in shared memory before any of them is
 // written, so source and destination rows may overlap.  Bit-exact 16-byte moves.
+#include "host_checks.h"
 #include "kernels.h"
 
 namespace jup {
@@ -30,7 +31,7 @@ __global__ void __launch_bounds__(128) kv_compact_kernel(CompactParams p) {
   const int pos = p.d_pos[b];
   int n = p.d_n_accept[b];
   n = n < 0 ? 0 : (n > p.q_len ? p.q_len : n);
-  if (pos < 0 || pos + p.q_len > p.capacity) return;  // never form an address outside the cache
+  if (pos < 0 || pos > p.capacity - p.q_len) return;  // never form an address outside the cache (no overflow: q_len <= capacity)
   if (threadIdx.x < n) {
     const int a = p.d_accept[b * p.q_len + threadIdx.x];
     src_row[threadIdx.x] = (a >= 0 && a < p.q_len) ? a : -1;  // an index outside the block moves nothing
@@ -70,12 +71,12 @@ cudaError_t launch_kv_compact(const CacheView& c, int q_len, const int32_t* d_po
   p.capacity = c.capacity;
   p.q_len = q_len;
   p.chunks = c.head_dim / 8;
-  static bool attr_done = false;
-  if (!attr_done) {
+  static PerDeviceOnce attr_done;
+  if (!attr_done.done()) {
     cudaError_t e = cudaFuncSetAttribute(kv_compact_kernel, cudaFuncAttributePreferredSharedMemoryCarveout,
                                          cudaSharedmemCarveoutMaxShared);
     if (e != cudaSuccess) return e;
-    attr_done = true;
+    attr_done.set();
   }
   li.launches += 1;
   return launch_pdl(kv_compact_kernel, dim3(static_cast<unsigned>(c.batch) * c.kv_heads), dim3(128), 0, st, p);

@@ -3,6 +3,7 @@
 // path: any head_dim in {64,128}, any pos / q_len.  One CTA = 64 chunk rows of
 // one (sequence, query head); heaviest row tiles are scheduled first.
 #include "attn_mma.cuh"
+#include "host_checks.h"
 #include "kernels.h"
 
 namespace jup {
@@ -88,26 +89,26 @@ cudaError_t launch_prefill_mma(const bf16* q, const CacheView& c, int q_heads, i
   cudaError_t e;
   if (c.head_dim == 128) {
     constexpr int smem = MmaTileCfg<128, 2>::SMEM_BYTES;
-    static bool attr_done = false;
-    if (!attr_done) {
+    static PerDeviceOnce attr_done;
+    if (!attr_done.done()) {
       e = cudaFuncSetAttribute(prefill_mma_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
       if (e == cudaSuccess)
         e = cudaFuncSetAttribute(prefill_mma_kernel<128>, cudaFuncAttributePreferredSharedMemoryCarveout,
                                  cudaSharedmemCarveoutMaxShared);
       if (e != cudaSuccess) return e;
-      attr_done = true;
+      attr_done.set();
     }
     prefill_mma_kernel<128><<<grid, 128, smem, st>>>(p);
   } else {
     constexpr int smem = MmaTileCfg<64, 2>::SMEM_BYTES;
-    static bool attr_done = false;
-    if (!attr_done) {
+    static PerDeviceOnce attr_done;
+    if (!attr_done.done()) {
       e = cudaFuncSetAttribute(prefill_mma_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
       if (e == cudaSuccess)
         e = cudaFuncSetAttribute(prefill_mma_kernel<64>, cudaFuncAttributePreferredSharedMemoryCarveout,
                                  cudaSharedmemCarveoutMaxShared);
       if (e != cudaSuccess) return e;
-      attr_done = true;
+      attr_done.set();
     }
     prefill_mma_kernel<64><<<grid, 128, smem, st>>>(p);
   }

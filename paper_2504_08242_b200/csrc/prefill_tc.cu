@@ -18,8 +18,13 @@
 // accumulators from TMEM and writing half of the output columns.
 // All mbarrier waits are bounded; on expiry the CTA sets the status word, drains its own
 // copies and MMAs, frees TMEM and returns.
+#include "host_checks.h"
+#include <atomic>
+
 #include "kernels.h"
 #include "tc_common.cuh"
+#include "tc_softmax.cuh"
+#include "tmap.h"
 
 namespace jup {
 
@@ -28,7 +33,6 @@ constexpr int TC_BM = 128;              // query rows per tile
 constexpr int TC_BN = 128;              // keys per KV tile
 constexpr int TC_TILE_BYTES = 32768;    // 128 x 128 bf16
 constexpr int TC_PANEL_BYTES = 16384;   // 128 rows x 64 elements
-constexpr float TC_RESCALE_THRESHOLD = 8.f;  // log2 units
 constexpr int TC_CLUSTER_MIN_TILES = 18;     // shortest KV walk (in tiles) that a cluster of 4 CTAs shares
 
 struct TcParams {
@@ -86,14 +90,6 @@ enum {
   BAR_COUNT = 24
 };
 
-// Output staging for a tiled store: a box of 128 rows x 32 fp32 (128-byte rows, 16-byte chunks XOR-swizzled by
-// the row as the 128-byte swizzle of the tensor map expects; conflict-free for one thread per row).
-__device__ __forceinline__ void stage_box_row(float* box, int r, const float (&v)[32]) {
-#pragma unroll
-  for (int cc = 0; cc < 8; ++cc)
-    *reinterpret_cast<float4*>(box + r * 32 + ((cc ^ (r & 7)) << 2)) =
-        make_float4(v[4 * cc], v[4 * cc + 1], v[4 * cc + 2], v[4 * cc + 3]);
-}
 constexpr int TC_BOX_FLOATS = TC_BM * 32;  // 16 KB
 
 // CL > 1: a thread-block cluster of CL CTAs shares one pair of query tiles; CTA r takes the KV tiles
@@ -385,106 +381,10 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
       const int nvalid = g < Tp ? p.prefix_len - g * TC_BN : lim - (g - Tp) * TC_BN;
       // warp-uniform flag, so the warp stays converged for the collective tcgen05 operations
       const bool masked = __any_sync(0xffffffffu, nvalid < TC_BN);
-      // ---- pass 1 over the S row: maximum (eight independent chains of 3-input max)
-      float mx;
-      {
-        float a[8];
-#pragma unroll
-        for (int k = 0; k < 8; ++k) a[k] = -INFINITY;
-#pragma unroll
-        for (int h2 = 0; h2 < 2; ++h2) {
-          uint32_t r0[32], r1[32];
-          tmem_ld32(tS + h2 * 64, r0);
-          tmem_ld32(tS + h2 * 64 + 32, r1);
-          tc_wait_ld();
-          if (masked) {
-#pragma unroll
-            for (int i = 0; i < 32; ++i) {
-              if (h2 * 64 + i >= nvalid) r0[i] = 0xff800000u;  // -inf
-              if (h2 * 64 + 32 + i >= nvalid) r1[i] = 0xff800000u;
-            }
-          }
-#pragma unroll
-          for (int i = 0; i < 32; i += 16)
-#pragma unroll
-            for (int k = 0; k < 8; ++k) {
-              a[k] = fmax3(a[k], __uint_as_float(r0[i + 2 * k]), __uint_as_float(r0[i + 2 * k + 1]));
-              a[k] = fmax3(a[k], __uint_as_float(r1[i + 2 * k]), __uint_as_float(r1[i + 2 * k + 1]));
-            }
-        }
-        mx = fmax3(fmax3(a[0], a[1], a[2]), fmax3(a[3], a[4], a[5]), fmaxf(a[6], a[7]));
-      }
-      const float mxs = mx * c;
-      // lazy rescale: the reference maximum only moves when the true maximum outgrew it by 2^8
-      // (in the partial modes a stream can meet rows that see none of its tile: the reference stays -inf,
-      // P is 0, and the first visible score moves it because -inf + 8 is still -inf)
-      const bool grow = PARTIAL ? (mxs > m_ref + TC_RESCALE_THRESHOLD)
-                              : ((j == 0) || (mxs > m_ref + TC_RESCALE_THRESHOLD));
-      bool o_waited = false;
-      if (j > 0 && __any_sync(0xffffffffu, grow)) {
-        const float alpha = grow ? fast_exp2(m_ref - mxs) : 1.f;
-        l *= alpha;
-        // O(j-1) must be complete before it is rescaled
-        ok = mbar_wait(bar(BAR_O_READY + x), (j - 1) & 1, abort_flag, p.status);
-        if (!ok) break;
-        o_waited = true;
-        tc_fence_after();
-#pragma unroll
-        for (int q4 = 0; q4 < 4; ++q4) {
-          uint32_t o[32];
-          tmem_ld32(tO + q4 * 32, o);
-          tc_wait_ld();
-#pragma unroll
-          for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
-          tmem_st32(tO + q4 * 32, o);
-        }
-      }
-      if (grow) m_ref = mxs;
-      // ---- pass 2: P = exp2(s*c - m_ref) as bf16 pairs, written in place over S (P column k holds
-      // keys 2k, 2k+1, so the writes stay behind the reads).  fp32-pair arithmetic, four row-sum chains,
-      // the next 32 columns are in flight while the current 32 are processed.
-      const float nm = (PARTIAL && m_ref == -INFINITY) ? 0.f : -m_ref;
-      const uint64_t c2 = pack2(c, c), nm2 = pack2(nm, nm);
-      uint64_t lacc[4];
-#pragma unroll
-      for (int k = 0; k < 4; ++k) lacc[k] = pack2(0.f, 0.f);
-      uint32_t sb[2][32];
-      tmem_ld32(tS, sb[0]);
-#pragma unroll
-      for (int q4 = 0; q4 < 4; ++q4) {
-        tc_wait_ld();
-        if (q4 < 3) tmem_ld32(tS + (q4 + 1) * 32, sb[(q4 + 1) & 1]);
-        uint32_t(&sv)[32] = sb[q4 & 1];
-        if (masked) {
-#pragma unroll
-          for (int i = 0; i < 32; ++i)
-            if (q4 * 32 + i >= nvalid) sv[i] = 0xff800000u;
-        }
-        uint32_t pk[16];
-#pragma unroll
-        for (int i = 0; i < 16; ++i) {
-          const uint64_t x = fma2(pack2(__uint_as_float(sv[2 * i]), __uint_as_float(sv[2 * i + 1])), c2, nm2);
-          float x0, x1;
-          unpack2(x, x0, x1);
-          const float p0 = fast_exp2(x0), p1 = fast_exp2(x1);
-          lacc[i & 3] = add2(lacc[i & 3], pack2(p0, p1));
-          pk[i] = pack_bf16(p0, p1);
-        }
-        tmem_st16(tS + q4 * 16, pk);
-      }
-      {
-        float a0, a1, b0, b1;
-        unpack2(add2(lacc[0], lacc[1]), a0, a1);
-        unpack2(add2(lacc[2], lacc[3]), b0, b1);
-        l += (a0 + a1) + (b0 + b1);
-      }
-      tc_wait_st();
-      // every phase of O_READY is waited on exactly once, in order, so a parity never aliases;
-      // PV(j) queues behind PV(j-1) in the tensor pipe anyway, so this costs no overlap
-      if (j > 0 && !o_waited) {
-        ok = mbar_wait(bar(BAR_O_READY + x), (j - 1) & 1, abort_flag, p.status);
-        if (!ok) break;
-      }
+      ok = softmax_tile_step<PARTIAL>(tS, tO, j, masked, ColumnLimit{nvalid}, c, m_ref, l, [&] {
+        return mbar_wait(bar(BAR_O_READY + x), (j - 1) & 1, abort_flag, p.status);
+      });
+      if (!ok) break;
       tc_fence_before();
       mbar_arrive(bar(BAR_P_FULL + x));
     }
@@ -718,57 +618,21 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
 
 // ---------------------------------------------------------------- host side
 
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-static EncodeTiledFn encode_fn() {
-  static EncodeTiledFn fn = nullptr;
-  static bool tried = false;
-  if (!tried) {
-    tried = true;
-    void* ptr = nullptr;
-    cudaDriverEntryPointQueryResult qres;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
-        qres == cudaDriverEntryPointSuccess)
-      fn = reinterpret_cast<EncodeTiledFn>(ptr);
-  }
-  return fn;
-}
-
-// 4-D bf16 tensor map with 64-element (128-byte) swizzled inner box.
-static bool make_map(CUtensorMap* m, const void* base, const uint64_t dims[4], const uint64_t strides_bytes[3],
-                     const uint32_t box[4]) {
-  EncodeTiledFn fn = encode_fn();
-  if (!fn) return false;
-  cuuint64_t gd[4] = {dims[0], dims[1], dims[2], dims[3]};
-  cuuint64_t gs[3];
-  for (int i = 0; i < 3; ++i) {
-    gs[i] = strides_bytes[i] ? strides_bytes[i] : 16;  // extent-1 dimensions may carry any stride
-    if (gs[i] % 16 || gs[i] >= (1ull << 40)) return false;
-  }
-  cuuint32_t bx[4] = {box[0], box[1], box[2], box[3]};
-  cuuint32_t es[4] = {1, 1, 1, 1};
-  return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), gd, gs, bx, es,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
 template <int NQ, bool SPLIT, int CL>
 static cudaError_t launch_variant(int64_t ctas, cudaStream_t st, const CUtensorMap& tq, const CUtensorMap& tk,
                                   const CUtensorMap& tv, const CUtensorMap& tpk, const CUtensorMap& tpv,
                                   const CUtensorMap& to, const CUtensorMap& tck, const CUtensorMap& tcv,
                                   const TcParams& p) {
   using Cfg = TcCfg<NQ, SPLIT>;
-  static bool done = false;
-  if (!done) {
+  static PerDeviceOnce done;
+  if (!done.done()) {
     cudaError_t e =
         cudaFuncSetAttribute(prefill_tc_kernel<NQ, SPLIT, CL>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM_BYTES);
     if (e == cudaSuccess)
       e = cudaFuncSetAttribute(prefill_tc_kernel<NQ, SPLIT, CL>, cudaFuncAttributePreferredSharedMemoryCarveout,
                                cudaSharedmemCarveoutMaxShared);
     if (e != cudaSuccess) return e;
-    done = true;
+    done.set();
   }
   return launch_pdl_cluster(prefill_tc_kernel<NQ, SPLIT, CL>, dim3(static_cast<unsigned>(ctas * CL)),
                             dim3(Cfg::THREADS), Cfg::SMEM_BYTES, st, static_cast<unsigned>(CL), tq, tk, tv, tpk, tpv, to, tck,
@@ -778,30 +642,33 @@ static cudaError_t launch_variant(int64_t ctas, cudaStream_t st, const CUtensorM
 // How many clusters of CL CTAs of the cluster-mode kernel can be resident at once (0 if the query fails).
 template <int CL>
 static int max_resident_clusters() {
-  static int n = -1;
-  if (n < 0) {
-    using Cfg = TcCfg<2, false>;
-    n = 0;
-    if (cudaFuncSetAttribute(prefill_tc_kernel<2, false, CL>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             Cfg::SMEM_BYTES) == cudaSuccess) {
-      cudaLaunchConfig_t cfg = {};
-      cfg.gridDim = dim3(CL * 64);
-      cfg.blockDim = dim3(Cfg::THREADS);
-      cfg.dynamicSmemBytes = Cfg::SMEM_BYTES;
-      cudaLaunchAttribute attr[1];
-      attr[0].id = cudaLaunchAttributeClusterDimension;
-      attr[0].val.clusterDim.x = CL;
-      attr[0].val.clusterDim.y = 1;
-      attr[0].val.clusterDim.z = 1;
-      cfg.attrs = attr;
-      cfg.numAttrs = 1;
-      int got = 0;
-      if (cudaOccupancyMaxActiveClusters(&got, prefill_tc_kernel<2, false, CL>, &cfg) == cudaSuccess) n = got;
-      else (void)cudaGetLastError();
-    } else {
-      (void)cudaGetLastError();
-    }
+  static std::atomic<int> cache[64];  // per device: 0 = not asked yet, else answer + 1
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 0;
+  const int cached = cache[dev].load(std::memory_order_acquire);
+  if (cached > 0) return cached - 1;
+  using Cfg = TcCfg<2, false>;
+  int n = 0;
+  if (cudaFuncSetAttribute(prefill_tc_kernel<2, false, CL>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           Cfg::SMEM_BYTES) == cudaSuccess) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(CL * 64);
+    cfg.blockDim = dim3(Cfg::THREADS);
+    cfg.dynamicSmemBytes = Cfg::SMEM_BYTES;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = CL;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    int got = 0;
+    if (cudaOccupancyMaxActiveClusters(&got, prefill_tc_kernel<2, false, CL>, &cfg) == cudaSuccess) n = got;
+    else (void)cudaGetLastError();
+  } else {
+    (void)cudaGetLastError();
   }
+  cache[dev].store(n + 1, std::memory_order_release);
   return n;
 }
 
@@ -817,18 +684,14 @@ static cudaError_t launch_tc(const bf16* q, const CacheView& c, const CacheView*
                              int pos, float scale, float* out, float* lse, int* status, void* workspace,
                              size_t workspace_bytes, cudaStream_t st, LaunchInfo& li) {
   CUtensorMap tq, tk, tv, tpk, tpv, to, tck, tcv;
+  if (!encode_fn()) return cudaErrorInvalidValue;
   {  // out: [batch][q_len][q_heads][128] fp32, boxes of 128 rows x 32 columns
-    EncodeTiledFn fn = encode_fn();
-    if (!fn) return cudaErrorInvalidValue;
-    cuuint64_t gd[4] = {TC_D, static_cast<cuuint64_t>(q_heads), static_cast<cuuint64_t>(q_len),
-                        static_cast<cuuint64_t>(c.batch)};
-    cuuint64_t gs[3] = {TC_D * 4ull, static_cast<cuuint64_t>(q_heads) * TC_D * 4ull,
-                        static_cast<cuuint64_t>(q_len) * q_heads * TC_D * 4ull};
-    cuuint32_t bx[4] = {32, 1, TC_BM, 1};
-    cuuint32_t es[4] = {1, 1, 1, 1};
-    if (fn(&to, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, out, gd, gs, bx, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
-           CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
-      return cudaErrorInvalidValue;
+    const uint64_t d[4] = {TC_D, static_cast<uint64_t>(q_heads), static_cast<uint64_t>(q_len),
+                           static_cast<uint64_t>(c.batch)};
+    const uint64_t s[3] = {TC_D * 4ull, static_cast<uint64_t>(q_heads) * TC_D * 4ull,
+                           static_cast<uint64_t>(q_len) * q_heads * TC_D * 4ull};
+    const uint32_t bx[4] = {32, 1, TC_BM, 1};
+    if (!make_map_f32(&to, out, d, s, bx)) return cudaErrorInvalidValue;
   }
   const uint64_t rows_valid = static_cast<uint64_t>(pos) + q_len;  // rows above are dead: TMA zero-fills them
   {
@@ -837,14 +700,14 @@ static cudaError_t launch_tc(const bf16* q, const CacheView& c, const CacheView*
     const uint64_t s[3] = {TC_D * 2ull, static_cast<uint64_t>(q_heads) * TC_D * 2ull,
                            static_cast<uint64_t>(q_len) * q_heads * TC_D * 2ull};
     const uint32_t bx[4] = {64, 1, TC_BM, 1};
-    if (!make_map(&tq, q, d, s, bx)) return cudaErrorInvalidValue;
+    if (!make_map_bf16(&tq, q, d, s, bx)) return cudaErrorInvalidValue;
   }
   {
     const uint64_t d[4] = {TC_D, rows_valid, static_cast<uint64_t>(c.kv_heads), static_cast<uint64_t>(c.batch)};
     const uint64_t s[3] = {static_cast<uint64_t>(c.sr) * 2, static_cast<uint64_t>(c.sh) * 2,
                            static_cast<uint64_t>(c.sb) * 2};
     const uint32_t bx[4] = {64, TC_BN, 1, 1};
-    if (!make_map(&tk, c.k, d, s, bx) || !make_map(&tv, c.v, d, s, bx)) return cudaErrorInvalidValue;
+    if (!make_map_bf16(&tk, c.k, d, s, bx) || !make_map_bf16(&tv, c.v, d, s, bx)) return cudaErrorInvalidValue;
   }
   if (prefix && prefix_len > 0) {  // rows at or beyond prefix_len are zero-filled by TMA
     const uint64_t d[4] = {TC_D, static_cast<uint64_t>(prefix_len), static_cast<uint64_t>(prefix->kv_heads),
@@ -852,7 +715,7 @@ static cudaError_t launch_tc(const bf16* q, const CacheView& c, const CacheView*
     const uint64_t s[3] = {static_cast<uint64_t>(prefix->sr) * 2, static_cast<uint64_t>(prefix->sh) * 2,
                            static_cast<uint64_t>(prefix->sb) * 2};
     const uint32_t bx[4] = {64, TC_BN, 1, 1};
-    if (!make_map(&tpk, prefix->k, d, s, bx) || !make_map(&tpv, prefix->v, d, s, bx)) return cudaErrorInvalidValue;
+    if (!make_map_bf16(&tpk, prefix->k, d, s, bx) || !make_map_bf16(&tpv, prefix->v, d, s, bx)) return cudaErrorInvalidValue;
   } else {
     tpk = tk;  // never dereferenced when there is no prefix
     tpv = tv;
@@ -877,7 +740,7 @@ static cudaError_t launch_tc(const bf16* q, const CacheView& c, const CacheView*
     const uint64_t s[3] = {static_cast<uint64_t>(copy_dst->sr) * 2, static_cast<uint64_t>(copy_dst->sh) * 2,
                            static_cast<uint64_t>(copy_dst->sb) * 2};
     const uint32_t bx[4] = {64, TC_BN, 1, 1};
-    if (!make_map(&tck, copy_dst->k, d, s, bx) || !make_map(&tcv, copy_dst->v, d, s, bx)) return cudaErrorInvalidValue;
+    if (!make_map_bf16(&tck, copy_dst->k, d, s, bx) || !make_map_bf16(&tcv, copy_dst->v, d, s, bx)) return cudaErrorInvalidValue;
   }
   p.out = out;
   p.lse = lse;

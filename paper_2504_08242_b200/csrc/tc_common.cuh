@@ -41,7 +41,8 @@ __device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
 // common tear-down.  Pass abort_flag = a private zero and status = nullptr for an unconditional
 // bounded wait.
 constexpr long long kWaitLimitCycles = 2000000000ll;
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status,
+                                          long long limit_cycles = kWaitLimitCycles) {
   if (mbar_test_wait(bar, parity)) return true;
   const long long t0 = clock64();
   for (uint32_t it = 1;; ++it) {
@@ -52,7 +53,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
         *abort_flag = 1;
         return false;
       }
-      if (clock64() - t0 > kWaitLimitCycles) break;
+      if (clock64() - t0 > limit_cycles) break;
     }
   }
   *abort_flag = 1;

@@ -1,0 +1,137 @@
+// One online-softmax step of the tcgen05 attention kernels: a thread owns one query row (one TMEM lane) and
+// walks the 128 fp32 scores of the current key tile twice with tcgen05.ld -- first the masked row maximum
+// (eight independent chains of 3-input max), then P = exp2(s * c - m) with fp32-pair arithmetic, written back in
+// place as bf16 pairs (P column k holds keys 2k and 2k + 1, so the writes stay behind the reads; the next 32
+// columns are in flight while the current 32 are processed).  The running sum stays in fp32 and the
+// accumulator O is rescaled lazily, only when the row maximum outgrew the reference by more than 2^8.
+#pragma once
+#include "tc_common.cuh"
+
+namespace jup {
+
+constexpr float TC_RESCALE_THRESHOLD = 8.f;  // log2 units
+
+// Visibility of the tile's columns to this thread's row (only consulted on tiles flagged as masked).
+struct ColumnLimit {  // columns [0, nvalid) are visible
+  int nvalid;
+  __device__ __forceinline__ bool operator()(int col) const { return col < nvalid; }
+};
+struct ColumnBits {  // bit (col & 31) of w[col >> 5] set: visible
+  uint32_t w[4];
+  __device__ __forceinline__ bool operator()(int col) const { return (w[col >> 5] >> (col & 31)) & 1u; }
+};
+
+// tS / tO: TMEM addresses (lane base included) of the row's 128 scores and of its 128 accumulator columns.
+// j: number of tiles this stream has processed before (0: O holds nothing yet).
+// masked: warp-uniform; when false every column is visible and `allow` is not consulted.
+// PARTIAL: the stream may meet rows that see none of a tile (their reference maximum stays -inf and P is 0).
+// wait_o(): waits until O(j-1) is complete (called exactly once when j > 0); returns false if the wait gave up,
+// and then so does this function.  On return P is complete in TMEM (tcgen05.wait::st done); the caller fences
+// and signals the MMA issuer.
+template <bool PARTIAL, class Allow, class WaitO>
+__device__ __forceinline__ bool softmax_tile_step(uint32_t tS, uint32_t tO, int j, bool masked, const Allow& allow,
+                                                  float c, float& m_ref, float& l, WaitO&& wait_o) {
+  // ---- pass 1: row maximum
+  float mx;
+  {
+    float a[8];
+#pragma unroll
+    for (int k = 0; k < 8; ++k) a[k] = -INFINITY;
+#pragma unroll
+    for (int h2 = 0; h2 < 2; ++h2) {
+      uint32_t r0[32], r1[32];
+      tmem_ld32(tS + h2 * 64, r0);
+      tmem_ld32(tS + h2 * 64 + 32, r1);
+      tc_wait_ld();
+      if (masked) {
+#pragma unroll
+        for (int i = 0; i < 32; ++i) {
+          if (!allow(h2 * 64 + i)) r0[i] = 0xff800000u;  // -inf
+          if (!allow(h2 * 64 + 32 + i)) r1[i] = 0xff800000u;
+        }
+      }
+#pragma unroll
+      for (int i = 0; i < 32; i += 16)
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+          a[k] = fmax3(a[k], __uint_as_float(r0[i + 2 * k]), __uint_as_float(r0[i + 2 * k + 1]));
+          a[k] = fmax3(a[k], __uint_as_float(r1[i + 2 * k]), __uint_as_float(r1[i + 2 * k + 1]));
+        }
+    }
+    mx = fmax3(fmax3(a[0], a[1], a[2]), fmax3(a[3], a[4], a[5]), fmaxf(a[6], a[7]));
+  }
+  const float mxs = mx * c;
+  // lazy rescale: the reference maximum only moves when the true maximum outgrew it by 2^8 (a row that has seen
+  // nothing keeps -inf, and its first visible score moves it because -inf + 8 is still -inf)
+  const bool grow = PARTIAL ? (mxs > m_ref + TC_RESCALE_THRESHOLD) : ((j == 0) || (mxs > m_ref + TC_RESCALE_THRESHOLD));
+  bool o_waited = false;
+  if (j > 0 && __any_sync(0xffffffffu, grow)) {
+    const float alpha = grow ? fast_exp2(m_ref - mxs) : 1.f;
+    l *= alpha;
+    if (!wait_o()) return false;  // O(j-1) must be complete before it is rescaled
+    o_waited = true;
+    tc_fence_after();
+#pragma unroll
+    for (int q4 = 0; q4 < 4; ++q4) {
+      uint32_t o[32];
+      tmem_ld32(tO + q4 * 32, o);
+      tc_wait_ld();
+#pragma unroll
+      for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
+      tmem_st32(tO + q4 * 32, o);
+    }
+  }
+  if (grow) m_ref = mxs;
+  // ---- pass 2: P
+  const float nm = (PARTIAL && m_ref == -INFINITY) ? 0.f : -m_ref;
+  const uint64_t c2 = pack2(c, c), nm2 = pack2(nm, nm);
+  uint64_t lacc[4];
+#pragma unroll
+  for (int k = 0; k < 4; ++k) lacc[k] = pack2(0.f, 0.f);
+  uint32_t sb[2][32];
+  tmem_ld32(tS, sb[0]);
+#pragma unroll
+  for (int q4 = 0; q4 < 4; ++q4) {
+    tc_wait_ld();
+    if (q4 < 3) tmem_ld32(tS + (q4 + 1) * 32, sb[(q4 + 1) & 1]);
+    uint32_t(&sv)[32] = sb[q4 & 1];
+    if (masked) {
+#pragma unroll
+      for (int i = 0; i < 32; ++i)
+        if (!allow(q4 * 32 + i)) sv[i] = 0xff800000u;
+    }
+    uint32_t pk[16];
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+      const uint64_t x = fma2(pack2(__uint_as_float(sv[2 * i]), __uint_as_float(sv[2 * i + 1])), c2, nm2);
+      float x0, x1;
+      unpack2(x, x0, x1);
+      const float p0 = fast_exp2(x0), p1 = fast_exp2(x1);
+      lacc[i & 3] = add2(lacc[i & 3], pack2(p0, p1));
+      pk[i] = pack_bf16(p0, p1);
+    }
+    tmem_st16(tS + q4 * 16, pk);
+  }
+  {
+    float a0, a1, b0, b1;
+    unpack2(add2(lacc[0], lacc[1]), a0, a1);
+    unpack2(add2(lacc[2], lacc[3]), b0, b1);
+    l += (a0 + a1) + (b0 + b1);
+  }
+  tc_wait_st();
+  // every phase of the O-complete barrier is waited on exactly once, in order, so a parity never aliases;
+  // PV(j) queues behind PV(j-1) in the tensor pipe anyway, so this costs no overlap
+  if (j > 0 && !o_waited && !wait_o()) return false;
+  return true;
+}
+
+// Output staging for a tiled store: a box of 128 rows x 32 fp32 (128-byte rows, 16-byte chunks XOR-swizzled by
+// the row as the 128-byte swizzle of the tensor map expects; conflict-free for one thread per row).
+__device__ __forceinline__ void stage_box_row(float* box, int r, const float (&v)[32]) {
+#pragma unroll
+  for (int cc = 0; cc < 8; ++cc)
+    *reinterpret_cast<float4*>(box + r * 32 + ((cc ^ (r & 7)) << 2)) =
+        make_float4(v[4 * cc], v[4 * cc + 1], v[4 * cc + 2], v[4 * cc + 3]);
+}
+
+}  // namespace jup
