@@ -198,13 +198,16 @@ class PrefillRun:
 
 
 class BranchRun:
-    """Device state and step function of a branch-attention workload.  `copies` > 1 rotates the
-    decode steps over independent copies of the caches so that each step reads cold data."""
+    """Device state and step function of a branch-attention workload.  `copies` > 1 rotates the launches over
+    independent copies of the caches so that each launch reads cold data.  A workload with a single decode step
+    (speculative verification) runs that step `passes` times per benchmark step, each pass on the next copy: the
+    data of every pass is cold (the copies together exceed L2 and L2 is flushed between steps) while the kernel's
+    code, as in a real decoding loop, is not fetched from DRAM for every launch."""
 
-    def __init__(self, ctx, w, device, copies=1):
+    def __init__(self, ctx, w, device, copies=1, passes=1):
         import torch
         import paper_2504_08242_b200 as J
-        self.ctx, self.w, self.copies = ctx, w, copies
+        self.ctx, self.w, self.copies, self.passes = ctx, w, copies, passes
         pk, pv, sk, sv = w.make_caches()
         self.caches = []
         for _ in range(copies):
@@ -220,15 +223,23 @@ class BranchRun:
                 q=_dev(q, device), k=_dev(kn, device), v=_dev(vn, device),
                 pos=torch.from_numpy(pos.astype(np.int32)).to(device),
                 lens=torch.from_numpy(lens.astype(np.int32)).to(device), max_len=int(lens.max())))
-            self.bytes += w.step_bytes(lens)
-            self.flops += w.step_flops(lens)
+            self.bytes += passes * w.step_bytes(lens)
+            self.flops += passes * w.step_flops(lens)
         self.out = torch.empty(w.n_branches, w.q_len, w.q_heads, w.head_dim, dtype=torch.float32, device=device)
         self.attn_events = None
 
+    def calls(self):
+        """(copy index, step data) of every library call of one benchmark step, in order."""
+        k = 0
+        for _ in range(self.passes):
+            for s in self.steps_data:
+                yield k % self.copies, s
+                k += 1
+
     def step(self):
         ctx, w, ev = self.ctx, self.w, self.attn_events
-        for t, s in enumerate(self.steps_data):
-            _, pdesc, sdesc = self.caches[t % self.copies]
+        for c, s in self.calls():
+            _, pdesc, sdesc = self.caches[c]
             if ev is not None:
                 import torch
                 a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -243,7 +254,15 @@ class BranchRun:
         return float(self.bytes)
 
     def attn_launches_per_step(self):
-        return len(self.steps_data)
+        return len(self.steps_data) * self.passes
+
+
+def branch_run(ctx, w, device, cold=True):
+    """The benchmark's form of a branch workload: launches rotate over cache copies that together exceed L2."""
+    if not cold:
+        return BranchRun(ctx, w, device, copies=1, passes=1)
+    copies = 8 if w.steps == 1 else 6
+    return BranchRun(ctx, w, device, copies=copies, passes=copies if w.steps == 1 else 1)
 
 
 def measure(run, steps, warmup, flush, barrier, use_graph=True, sampler=None):
@@ -374,15 +393,15 @@ def e2e_measure(run, steps, warmup, flush):
                                                                      c["pos"], w.scale, c["out"])),
                           (ho, c["out"])))
     else:
-        host = [(pin(s["q"]), pin(s["k"]), pin(s["v"]), pin(s["pos"]), pin(s["lens"])) for s in run.steps_data]
+        host = {id(s): (pin(s["q"]), pin(s["k"]), pin(s["v"]), pin(s["pos"]), pin(s["lens"])) for s in run.steps_data}
         ho = torch.empty(run.out.shape, dtype=torch.float32).pin_memory()
-        for hq, hk, hv, hp, hl in host:
-            h2d += hq.numel() * 2 + hk.numel() * 2 + hv.numel() * 2 + hp.numel() * 4 + hl.numel() * 4
-            d2h += ho.numel() * 4
         ctx, w = run.ctx, run.w
         calls = []
-        for t, (s, (hq, hk, hv, hp, hl)) in enumerate(zip(run.steps_data, host)):
-            _, pdesc, sdesc = run.caches[t % run.copies]
+        for c, s in run.calls():
+            hq, hk, hv, hp, hl = host[id(s)]
+            h2d += hq.numel() * 2 + hk.numel() * 2 + hv.numel() * 2 + hp.numel() * 4 + hl.numel() * 4
+            d2h += ho.numel() * 4
+            _, pdesc, sdesc = run.caches[c]
             calls.append((((s["q"], hq), (s["k"], hk), (s["v"], hv), (s["pos"], hp), (s["lens"], hl)),
                           (lambda s=s, pdesc=pdesc, sdesc=sdesc: ctx.branch_append_attn(
                               s["q"], s["k"], s["v"], pdesc, w.prefix_len, sdesc, s["lens"], s["max_len"], w.n_branches,
@@ -478,7 +497,7 @@ def config_of(name, w, extra=None):
     else:
         c = {"workload": name, "branches": w.n_branches, "q_heads": w.q_heads, "kv_heads": w.kv_heads,
              "head_dim": w.head_dim, "prefix_len": w.prefix_len, "suffix_history": [w.suffix_lo, w.suffix_hi],
-             "q_len": w.q_len, "decode_steps": w.steps, "calls_per_step": w.steps}
+             "q_len": w.q_len, "decode_steps": w.steps}
     c["l2"] = "flushed between steps (buffer of 2x L2 rewritten)"
     c["launch"] = "one CUDA-graph replay per step"
     if extra:
@@ -578,7 +597,7 @@ def main():
     w = make_workload(name)
     is_prefill = isinstance(w, synth.PrefillWorkload)
     # branch workloads fit in L2: rotate the decode steps over independent cache copies so each reads cold data
-    run = PrefillRun(ctx, w, device) if is_prefill else BranchRun(ctx, w, device, copies=6)
+    run = PrefillRun(ctx, w, device) if is_prefill else branch_run(ctx, w, device)
 
     sampler = ClockSampler(local_rank)
     sampler.start()
@@ -615,7 +634,8 @@ def main():
     line = {"metric": METRIC, "value": value, "unit": unit_of(w), "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-            "config": config_of(name, w, dict({} if is_prefill else {"cache_copies_rotated": run.copies},
+            "config": config_of(name, w, dict({} if is_prefill else {"cache_copies_rotated": run.copies, "passes_per_step": run.passes,
+                                                                    "calls_per_step": run.attn_launches_per_step()},
                                               **({"launch": "eager"} if args.no_graph else {}))),
             "clocks": clocks, "gpu_launches": m["launches_per_step"] * args.steps,
             "e2e": {"value": e2e_value, "unit": unit_of(w), "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
@@ -656,8 +676,8 @@ def other_workloads(ctx, device, flush, peaks, skip, run=None):
                          "attn_frac_of_bf16_sustained": ka / peaks["bf16_tflops_sustained"], "steps": steps}
         else:
             res = {}
-            for label, copies in (("cold", 6), ("warm", 1)):
-                r = BranchRun(ctx, w, device, copies=copies)
+            for label in ("cold", "warm"):
+                r = branch_run(ctx, w, device, cold=label == "cold")
                 m = measure(r, steps, 3, flush, lambda: None)
                 gb = r.units() / (m["attn_ms_per_step"] * 1e-3) / 1e9
                 res[label] = {"attn_gbs": gb, "frac_of_hbm_peak": gb / peaks["hbm_gbs"],

@@ -209,8 +209,8 @@ jupiter_status jupiter_branch_append_attn(jupiter_ctx* ctx, const void* q, const
  * query rows per kv head (decode), a tensor-core kernel (tcgen05 / TMEM) for many rows with head_dim 128, and a
  * general split-KV kernel.  This call pins the choice for later calls on `ctx`; JUPITER_BRANCH_AUTO restores the
  * default.  A call whose shape the pinned kernel cannot take returns JUPITER_ERR_UNSUPPORTED (the tensor-core
- * kernel needs head_dim 128, scale > 0, a group size q_heads / kv_heads that is a power of two, and
- * q_len * group >= 5).  All three give the same result up to rounding. */
+ * kernel needs head_dim 128, scale > 0, and either q_len * group <= 128 or a group size q_heads / kv_heads that
+ * divides 128).  All three give the same result up to rounding. */
 typedef enum {
   JUPITER_BRANCH_AUTO = 0,
   JUPITER_BRANCH_STREAM = 1,

@@ -3,32 +3,37 @@
 // point-extending requests share the prompt's KVCache).
 //
 // head_dim 128.  The stacked rows of a kv head -- (branch, draft token, head of the group), in that order -- are
-// cut into tiles of 128 rows.  A unit = (kv head, row tile).  Every row belongs to one branch and may see the shared
-// prefix plus that branch's suffix, so a row keeps ONE online-softmax state in its TMEM lane while the unit walks
+// cut into row tiles of at most 128 rows: whole branches while a branch has at most 128 rows (the same number
+// of branches in every tile, so that the tiles carry equal work), else 128-row slices of one branch.
+// A unit = (kv head, row tile).  Every row belongs to one branch and may see the shared prefix plus that
+// branch's suffix, so a row keeps ONE online-softmax state in its TMEM lane while the unit walks
 //     prefix | suffix of the tile's first branch | ... | suffix of its last branch
 // in tiles of 128 keys: a prefix tile is visible to every row, a suffix tile to the rows of its branch below
-// their causal limit (or tree mask).  A prefix K/V tile is therefore fetched once per 128 rows, not once per branch.
+// their causal limit (or tree mask).  A prefix K/V tile is therefore fetched once per row tile, not once per branch.
 //
-// `ctas_per_unit` CTAs share a unit: the prefix tiles are cut into equal contiguous ranges, one per CTA, and so
-// are the suffix tiles (the prefix share does not depend on the device-side lengths, so its first loads are in
-// flight while the lengths arrive).  Inside a CTA:
-//   loader warp  : TMA (tiled, 128-byte swizzle) Q once -- one box [128/G tokens][G heads][64] lands in stacked-row
-//                  order -- then the K/V tiles of the CTA's list into 3-stage rings
+// `ctas_per_unit` CTAs, a thread-block cluster, share a unit: the prefix tiles are cut into equal contiguous
+// ranges, one per CTA, and so are the suffix tiles (the prefix share does not depend on the device-side lengths,
+// so its first loads are in flight while the lengths arrive).  Inside a CTA:
+//   loader warp  : TMA (tiled, 128-byte swizzle) Q once -- one box [tokens][G heads][64] lands in stacked-row
+//                  order -- then the K/V tiles of the CTA's list into 3-stage rings, K and V refilled independently
 //   patch warp   : the last tiles of a branch's suffix hold rows that TMA cannot know about: rows at or beyond the
 //                  device-side length (dead; their V rows are zeroed so that 0 x NaN never reaches an accumulator)
 //                  and, with the fused KVCache write, the rows of this step's block, which are read from
-//                  k_new / v_new into the tile (and stored into the cache by the unit that owns the branch)
-//   MMA warp     : one thread issues tcgen05.mma  S = Q K^T  and  O += P V, accumulators in TMEM
+//                  k_new / v_new into the tile (and stored into the cache by the unit that owns them)
+//   MMA warp     : one thread issues tcgen05.mma  S = Q K^T  and  O += P V, accumulators in TMEM; it polls both
+//                  streams and the rings and never blocks on one of them
 //   softmax WGs  : two warpgroups run two independent online-softmax streams over the even and the odd tiles of
 //                  the CTA's list (one thread per row); a warp none of whose rows sees a tile only zeroes its P
 // TMEM (512 columns): S_0 | S_1 | O_0 | O_1.
-// At the end the two streams are merged.  With one CTA per unit the result is normalised and written with tiled
-// stores.  Otherwise the CTA writes its unnormalised partial (O, m, l) to scratch and takes a ticket on the
-// unit's counter; the CTA that takes the last ticket merges the unit's partials in CTA order (so the result
-// never depends on timing), puts the counter back to zero and writes the output.  Nothing waits on another CTA.
+// At the end the two streams of a CTA are merged in registers and every row's unnormalised (O, m, l) is pushed
+// into the shared memory of the CTA of the cluster that owns the row (distributed shared memory; the K/V rings are
+// free by then: one cluster barrier before the push says so, a second one after it says that every partial has
+// arrived).  The owner adds the partials in CTA order -- the result never depends on timing -- normalises and
+// writes the output rows.  No global scratch, no atomics, one launch.
 // All mbarrier waits are bounded; on expiry the CTA sets the status word, drains its own copies and MMAs,
-// frees TMEM and returns.
+// frees TMEM and returns (every thread still passes the cluster barriers).
 #include <algorithm>
+#include <atomic>
 
 #include "host_checks.h"
 #include "kernels.h"
@@ -39,23 +44,23 @@
 namespace jup {
 
 constexpr int BT_D = 128;
-constexpr int BT_BM = 128;             // stacked rows per tile
+constexpr int BT_BM = 128;             // stacked rows per tile (at most)
 constexpr int BT_BN = 128;             // keys per KV tile
 constexpr int BT_TILE_BYTES = 32768;   // 128 x 128 bf16
 constexpr int BT_PANEL_BYTES = 16384;  // 128 rows x 64 elements
 constexpr int BT_KV_STAGES = 3;
-constexpr int BT_MAX_TILES = 160;      // tiles one CTA can list
-constexpr int BT_MAX_BRANCHES = 32;    // branches with a row in one 128-row tile
-constexpr int BT_MAX_CTAS = 16;        // CTAs per unit
-constexpr int BT_BOX_FLOATS = BT_BM * 32;
-constexpr int BT_PART_FLOATS = BT_BM * BT_D;  // one CTA's partial accumulator
-constexpr int BT_ML_FLOATS = BT_BM * 2;       // and its (m, l) pairs
+constexpr int BT_MAX_BRANCHES = 32;    // branches in one row tile
+constexpr int BT_MAX_CTAS = 8;         // CTAs per unit (the portable cluster size)
+constexpr int BT_RECV_STRIDE = BT_D + 4;  // floats per received row: O, then (m, l), padded against bank conflicts
 
 struct BtParams {
   int n_branches, q_len, q_heads, group, kv_heads;
   int prefix_len, max_suffix_len;
-  int row_tiles;      // 128-row tiles per kv head
-  int ctas_per_unit;
+  int row_tiles;          // row tiles per kv head
+  int branches_per_tile;  // whole branches per row tile (slices_per_branch == 1)
+  int slices_per_branch;  // > 1: a branch has more than 128 rows and is cut into 128-row slices
+  int box_tokens;         // tokens in the Q box
+  int ctas_per_unit;      // cluster size
   float scale_log2;
   long long wait_limit;
   const int32_t* d_suffix_len;
@@ -65,24 +70,23 @@ struct BtParams {
   bf16* k_cache;              // the suffix cache (written only with the fused write)
   bf16* v_cache;
   int64_t sb, sh, sr;
+  float* out;
   float* lse;
   int* status;
-  int* counters;  // [units], zero on entry and on exit
-  float* part;    // [units][ctas_per_unit][32 column chunks][128 rows] float4
-  float* ml;      // [units][ctas_per_unit][128 rows] (m, l)
 };
 
-// shared memory: [Q][K ring][V ring][barriers, flags][lengths][tile table]
+// shared memory: [Q][K ring][V ring][barriers, flags][lengths and tile counts of the row tile's branches]
 constexpr int BT_SMEM_Q = 0;
 constexpr int BT_SMEM_K = BT_TILE_BYTES;
 constexpr int BT_SMEM_V = BT_SMEM_K + BT_KV_STAGES * BT_TILE_BYTES;
 constexpr int BT_SMEM_BAR = BT_SMEM_V + BT_KV_STAGES * BT_TILE_BYTES;
 constexpr int BT_SMEM_LEN = BT_SMEM_BAR + 256;
-constexpr int BT_SMEM_TABLE = BT_SMEM_LEN + 2 * BT_MAX_BRANCHES * 4;
-constexpr int BT_SMEM_BYTES = BT_SMEM_TABLE + BT_MAX_TILES * 4 + 1024;  // + slack for 1024-byte alignment
+constexpr int BT_SMEM_BYTES = BT_SMEM_LEN + 2 * BT_MAX_BRANCHES * 4 + 1024;  // + slack for 1024-byte alignment
 static_assert(BT_SMEM_BYTES <= 227 * 1024, "shared memory per CTA");
+// partials received from the cluster live in the K/V rings: [source CTA][row of the slice][BT_RECV_STRIDE]
+static_assert((BT_BM + BT_MAX_CTAS) * BT_RECV_STRIDE * 4 <= 2 * BT_KV_STAGES * BT_TILE_BYTES, "partials fit in the rings");
 constexpr int BT_LOADER_WARP = 8,  // warps 0..7: the two softmax warpgroups
-               BT_MMA_WARP = 9, BT_PATCH_WARP = 10;
+              BT_MMA_WARP = 9, BT_PATCH_WARP = 10;
 constexpr int BT_THREADS = 32 * 11;
 
 enum {
@@ -99,16 +103,24 @@ enum {
   BT_BAR_COUNT = 23
 };
 
-// tile table entry: bits [0,8) branch as an index into the tile's branches (0xff: shared prefix),
-// [8,24) tile number inside the segment, bit 24: the patch warp has work on it
-__device__ __forceinline__ int bt_seg(uint32_t e) { return static_cast<int>(e & 0xffu); }
-__device__ __forceinline__ int bt_tile(uint32_t e) { return static_cast<int>((e >> 8) & 0xffffu); }
-__device__ __forceinline__ bool bt_patch(uint32_t e) { return (e >> 24) & 1u; }
+// One entry of a CTA's tile list.
+struct BtTile {
+  int seg;     // branch as an index into the row tile's branches; -1: the shared prefix
+  int tile;    // tile number inside the segment
+  bool patch;  // the patch warp has work on it
+};
+
+__device__ __forceinline__ void st_cluster_v4(uint32_t addr, float a, float b, float c, float d) {
+  asm volatile("st.shared::cluster.v4.f32 [%0], {%1, %2, %3, %4};\n" ::"r"(addr), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
+}
+__device__ __forceinline__ void st_cluster_v2(uint32_t addr, float a, float b) {
+  asm volatile("st.shared::cluster.v2.f32 [%0], {%1, %2};\n" ::"r"(addr), "f"(a), "f"(b) : "memory");
+}
 
 __global__ void __launch_bounds__(BT_THREADS, 1)
 branch_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_pk,
                  const __grid_constant__ CUtensorMap tm_pv, const __grid_constant__ CUtensorMap tm_sk,
-                 const __grid_constant__ CUtensorMap tm_sv, const __grid_constant__ CUtensorMap tm_o, BtParams p) {
+                 const __grid_constant__ CUtensorMap tm_sv, BtParams p) {
   constexpr int KV_STAGES = BT_KV_STAGES;
   extern __shared__ unsigned char smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -117,24 +129,32 @@ branch_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
   const uint32_t sBar = smem_base + BT_SMEM_BAR;
   volatile int* abort_flag = reinterpret_cast<volatile int*>(smem_gen + BT_SMEM_BAR + 8 * BT_BAR_COUNT);
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem_gen + BT_SMEM_BAR + 8 * BT_BAR_COUNT + 8);
-  volatile int* n_tiles_slot = reinterpret_cast<volatile int*>(smem_gen + BT_SMEM_BAR + 8 * BT_BAR_COUNT + 16);
-  volatile int* last_slot = reinterpret_cast<volatile int*>(smem_gen + BT_SMEM_BAR + 8 * BT_BAR_COUNT + 24);
+  volatile int* suffix_share = reinterpret_cast<volatile int*>(smem_gen + BT_SMEM_BAR + 8 * BT_BAR_COUNT + 16);  // [2]
   int* len_s = reinterpret_cast<int*>(smem_gen + BT_SMEM_LEN);  // clamped suffix length of the tile's branches
   int* cum_s = len_s + BT_MAX_BRANCHES;                         // one past the last suffix tile of each
-  uint32_t* table = reinterpret_cast<uint32_t*>(smem_gen + BT_SMEM_TABLE);
   auto bar = [&](int i) { return sBar + 8u * i; };
   const long long wl = p.wait_limit;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int C = p.ctas_per_unit;
-  const int unit = blockIdx.x / C, crank = blockIdx.x % C;
+  const int unit = blockIdx.x / C, crank = blockIdx.x % C;  // clusters are consecutive CTAs: crank is the cluster rank
   const int rt = unit % p.row_tiles, hk = unit / p.row_tiles;
-  const int n = p.q_len, G = p.group, nG = n * G;
-  const int rows_total = p.n_branches * nG;
-  const int R0 = rt * BT_BM;
-  const int rows_here = min(BT_BM, rows_total - R0);
-  const int b_first = R0 / nG;
-  const int nb = (R0 + rows_here - 1) / nG - b_first + 1;  // branches with a row in this tile
+  const int n = p.q_len, G = p.group;
+  // ---- the row tile: tokens [tok0, tok0 + ntok) of the stacked (branch, draft row) order, all heads of the group
+  int b_first, nb, tok0, ntok;
+  if (p.slices_per_branch == 1) {
+    b_first = rt * p.branches_per_tile;
+    nb = min(p.branches_per_tile, p.n_branches - b_first);
+    tok0 = b_first * n;
+    ntok = nb * n;
+  } else {
+    b_first = rt / p.slices_per_branch;
+    nb = 1;
+    const int first = (rt % p.slices_per_branch) * (BT_BM / G);
+    tok0 = b_first * n + first;
+    ntok = min(BT_BM / G, n - first);
+  }
+  const int rows_here = ntok * G;
   const int P = p.prefix_len;
   const bool fused = p.k_new != nullptr;
   // this CTA's share of the prefix tiles: known without any memory access
@@ -158,7 +178,6 @@ branch_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
       tma_prefetch_desc(&tm_pk);
       tma_prefetch_desc(&tm_pv);
     }
-    tma_prefetch_desc(&tm_o);
   }
   tc_fence_before();
   __syncthreads();
@@ -166,14 +185,19 @@ branch_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
   const uint32_t tmem = *tmem_slot;
   pdl_wait();  // everything above overlapped the previous kernel's tail; global memory is touched from here on
 
-  auto load_tile = [&](int s, uint32_t e) {  // K and V of list entry e into the ring slot of sequence number s
+  auto load_k = [&](int s, const BtTile& e) {  // K of list entry e into the ring slot of sequence number s
     const int slot = s % KV_STAGES;
-    const bool pre = bt_seg(e) == 0xff;
-    const int row = bt_tile(e) * BT_BN, bb = pre ? 0 : b_first + bt_seg(e);
+    const bool pre = e.seg < 0;
+    const int row = e.tile * BT_BN, bb = pre ? 0 : b_first + e.seg;
     mbar_expect_tx(bar(BT_K_FULL + slot), BT_TILE_BYTES);
     const CUtensorMap* mk = pre ? &tm_pk : &tm_sk;
     tma_load_4d(sK + slot * BT_TILE_BYTES, mk, bar(BT_K_FULL + slot), 0, row, hk, bb);
     tma_load_4d(sK + slot * BT_TILE_BYTES + BT_PANEL_BYTES, mk, bar(BT_K_FULL + slot), 64, row, hk, bb);
+  };
+  auto load_v = [&](int s, const BtTile& e) {
+    const int slot = s % KV_STAGES;
+    const bool pre = e.seg < 0;
+    const int row = e.tile * BT_BN, bb = pre ? 0 : b_first + e.seg;
     mbar_expect_tx(bar(BT_V_FULL + slot), BT_TILE_BYTES);
     const CUtensorMap* mv = pre ? &tm_pv : &tm_sv;
     tma_load_4d(sV + slot * BT_TILE_BYTES, mv, bar(BT_V_FULL + slot), 0, row, hk, bb);
@@ -181,13 +205,18 @@ branch_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
   };
   const int pre_issued = min(npre, KV_STAGES);
   if (warp == BT_LOADER_WARP && lane == 0) {
-    // Q: token rows R0 / G .. of heads hk G .., one box per 64-column panel
-    mbar_expect_tx(bar(BT_Q_FULL), BT_TILE_BYTES);
-    tma_load_4d(sQ, &tm_q, bar(BT_Q_FULL), 0, hk * G, R0 / G, 0);
-    tma_load_4d(sQ + BT_PANEL_BYTES, &tm_q, bar(BT_Q_FULL), 64, hk * G, R0 / G, 0);
-    for (int s = 0; s < pre_issued; ++s) load_tile(s, 0xffu | (static_cast<uint32_t>(p0 + s) << 8));
+    // Q: box_tokens tokens from tok0 on, heads hk G .. hk G + G - 1, one box per 64-column panel; the box lands as
+    // rows (token, head) = stacked-row order.  Rows of the Q buffer beyond the box are never written: they belong
+    // to no row of this tile and whatever the tensor cores make of them is never used.
+    mbar_expect_tx(bar(BT_Q_FULL), static_cast<uint32_t>(p.box_tokens) * G * 256u);
+    tma_load_4d(sQ, &tm_q, bar(BT_Q_FULL), 0, hk * G, tok0, 0);
+    tma_load_4d(sQ + BT_PANEL_BYTES, &tm_q, bar(BT_Q_FULL), 64, hk * G, tok0, 0);
+    for (int s = 0; s < pre_issued; ++s) {
+      load_k(s, BtTile{-1, p0 + s, false});
+      load_v(s, BtTile{-1, p0 + s, false});
+    }
   } else if (warp == 0) {
-    // ---- tile list of this CTA: its prefix share, then its share of the suffix tiles of the tile's branches
+    // ---- lengths and tile counts of the row tile's branches
     int L = 0;
     if (lane < nb) {
       L = __ldg(p.d_suffix_len + b_first + lane);
@@ -201,75 +230,89 @@ branch_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
     }
     len_s[lane] = L;
     cum_s[lane] = cum;
-    const int Ts = __shfl_sync(0xffffffffu, cum, 31);
-    const int s0 = static_cast<int>(static_cast<int64_t>(Ts) * crank / C);
-    const int nsuf = static_cast<int>(static_cast<int64_t>(Ts) * (crank + 1) / C) - s0;
-    __syncwarp();
-    const int total = min(npre + nsuf, BT_MAX_TILES);  // the host sized the launch so that the list fits
-    for (int u = lane; u < total; u += 32) {
-      uint32_t e;
-      if (u < npre) {
-        e = 0xffu | (static_cast<uint32_t>(p0 + u) << 8);
-      } else {
-        const int g = s0 + u - npre;
-        int j = 0;
-        while (j < nb - 1 && cum_s[j] <= g) ++j;
-        const int tile = g - (j > 0 ? cum_s[j - 1] : 0);
-        const int first_special = fused ? len_s[j] - n : len_s[j];  // first row that is new or dead
-        const bool patch = (tile + 1) * BT_BN > first_special;
-        e = static_cast<uint32_t>(j) | (static_cast<uint32_t>(tile) << 8) | (patch ? 1u << 24 : 0u);
-      }
-      table[u] = e;
+    if (lane == 31) {  // this CTA's share of the unit's suffix tiles
+      const int s0 = static_cast<int>(static_cast<int64_t>(cum) * crank / C);
+      suffix_share[0] = s0;
+      suffix_share[1] = static_cast<int>(static_cast<int64_t>(cum) * (crank + 1) / C) - s0;
     }
-    if (lane == 0) *n_tiles_slot = total;
   }
   __syncthreads();
-  const int Tall = *n_tiles_slot;
+  const int s0 = suffix_share[0];
+  const int Tall = npre + suffix_share[1];
+  // Entry `s` of this CTA's list: its prefix share first, then its share of the suffix tiles of the row tile's
+  // branches.  A role walks the list in increasing order and keeps the branch it has reached in `cursor`.
+  auto tile_at = [&](int s, int& cursor) {
+    if (s < npre) return BtTile{-1, p0 + s, false};
+    const int g = s0 + (s - npre);
+    while (cursor < nb - 1 && cum_s[cursor] <= g) ++cursor;
+    const int tile = g - (cursor > 0 ? cum_s[cursor - 1] : 0);
+    const int first_special = fused ? len_s[cursor] - n : len_s[cursor];  // first row that is new or dead
+    return BtTile{cursor, tile, (tile + 1) * BT_BN > first_special};
+  };
   const int T[2] = {(Tall + 1) >> 1, Tall >> 1};  // stream x takes the sequence numbers 2 i + x
+
+  // a softmax thread's state after its last tile, kept for the merge behind the role branches
+  float fin_m = -INFINITY, fin_l = 0.f, fin_w_own = 0.f, fin_w_oth = 0.f;
 
   if (warp == BT_LOADER_WARP) {
     // =============================================================== loader
     if (lane == 0) {
+      // K and V rings are refilled independently: a K slot is free once its Q K^T has run, a V slot only after
+      // its P V, and neither queue may hold up the other
       bool ok = true;
-      int issued = pre_issued;
-      for (int s = pre_issued; s < Tall && ok; ++s) {
-        const int slot = s % KV_STAGES, u = s / KV_STAGES;
-        if (u > 0) {
-          ok = mbar_wait(bar(BT_K_EMPTY + slot), (u - 1) & 1, abort_flag, p.status, wl) &&
-               mbar_wait(bar(BT_V_EMPTY + slot), (u - 1) & 1, abort_flag, p.status, wl);
-          if (!ok) break;
+      int kn = pre_issued, vn = pre_issued, k_cursor = 0, v_cursor = 0;
+      PollGuard guard(wl);
+      while (ok && (kn < Tall || vn < Tall)) {
+        bool progress = false;
+        if (kn < Tall && (kn < KV_STAGES || mbar_test_wait(bar(BT_K_EMPTY + kn % KV_STAGES), (kn / KV_STAGES - 1) & 1))) {
+          load_k(kn, tile_at(kn, k_cursor));
+          ++kn;
+          progress = true;
         }
-        load_tile(s, table[s]);
-        issued = s + 1;
+        if (vn < Tall && (vn < KV_STAGES || mbar_test_wait(bar(BT_V_EMPTY + vn % KV_STAGES), (vn / KV_STAGES - 1) & 1))) {
+          load_v(vn, tile_at(vn, v_cursor));
+          ++vn;
+          progress = true;
+        }
+        if (progress) guard.progress();
+        else ok = guard.idle(abort_flag, p.status);
       }
       if (*abort_flag) {
         // wait (bounded) until every copy this thread started has landed before shared memory is released
         int dummy = 0;
         volatile int* none = &dummy;
-        for (int s = max(0, issued - KV_STAGES); s < issued; ++s) {
-          mbar_wait(bar(BT_K_FULL + s % KV_STAGES), (s / KV_STAGES) & 1, none, nullptr, wl);
-          mbar_wait(bar(BT_V_FULL + s % KV_STAGES), (s / KV_STAGES) & 1, none, nullptr, wl);
-        }
-        mbar_wait(bar(BT_Q_FULL), 0, none, nullptr, wl);
+        for (int s = max(0, kn - KV_STAGES); s < kn; ++s)
+          mbar_wait(bar(BT_K_FULL + s % KV_STAGES), (s / KV_STAGES) & 1, none, nullptr);
+        for (int s = max(0, vn - KV_STAGES); s < vn; ++s)
+          mbar_wait(bar(BT_V_FULL + s % KV_STAGES), (s / KV_STAGES) & 1, none, nullptr);
+        mbar_wait(bar(BT_Q_FULL), 0, none, nullptr);
       }
     }
     __syncwarp();
   } else if (warp == BT_PATCH_WARP) {
     // =============================================================== patch warp
     bool ok = true;
+    int cursor = 0;
     for (int s = 0; s < Tall && ok; ++s) {
       const int slot = s % KV_STAGES, u = s / KV_STAGES;
-      ok = mbar_wait(bar(BT_K_FULL + slot), u & 1, abort_flag, p.status, wl) &&
-           mbar_wait(bar(BT_V_FULL + slot), u & 1, abort_flag, p.status, wl);
+      // one lane spins; the others then observe the completed phases themselves (a single test each)
+      if (lane == 0)
+        ok = mbar_wait(bar(BT_K_FULL + slot), u & 1, abort_flag, p.status, wl) &&
+             mbar_wait(bar(BT_V_FULL + slot), u & 1, abort_flag, p.status, wl);
+      ok = __shfl_sync(0xffffffffu, ok, 0);
+      if (!ok) break;
+      if (lane != 0)
+        ok = mbar_wait(bar(BT_K_FULL + slot), u & 1, abort_flag, p.status, wl) &&
+             mbar_wait(bar(BT_V_FULL + slot), u & 1, abort_flag, p.status, wl);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
-      const uint32_t e = table[s];
-      if (bt_patch(e)) {
-        const int j = bt_seg(e), b = b_first + j, L = len_s[j], key0 = bt_tile(e) * BT_BN;
+      const BtTile e = tile_at(s, cursor);
+      if (e.patch) {
+        const int j = e.seg, b = b_first + j, L = len_s[j], key0 = e.tile * BT_BN;
         const int new_begin = fused ? L - n : L;
         const int r_begin = max(new_begin - key0, 0);
-        // the unit that holds the branch's first stacked row stores the block into the cache
-        const bool writer = fused && (b * nG) / BT_BM == rt;
+        // the block's rows go into the cache once per (branch, kv head): by the unit whose row tile starts the branch
+        const bool writer = fused && (p.slices_per_branch == 1 || rt % p.slices_per_branch == 0);
         const uint32_t kslot = sK + slot * BT_TILE_BYTES, vslot = sV + slot * BT_TILE_BYTES;
         for (int idx = lane; idx < (BT_BN - r_begin) * 16; idx += 32) {
           const int r = r_begin + (idx >> 4), c = idx & 15;
@@ -322,53 +365,55 @@ branch_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
           tc_mma_ts(o_col(x), s_col(x) + ks * 8, tc_smem_desc(vb + ks * 2048, BT_PANEL_BYTES, 1024), idesc_pv,
                     (!first || ks > 0));
       };
-      bool ok = true;
-      int ready = -1;  // tiles up to this sequence number have landed and are patched
-      auto need = [&](int s) {
-        while (ready < s && ok) {
+      // The issuer never blocks on one stream while the other has work: each pass looks at what has landed and at
+      // both streams' P, and issues whatever is ready.  Per stream the order is fixed: S(s) -> [softmax] -> P V(s)
+      // -> S(s + 2), because the stream has one S buffer.
+      bool ok = mbar_wait(bar(BT_Q_FULL), 0, abort_flag, p.status, wl);  // (also when the list is empty: the copy must land)
+      int ready = -1;                // tiles up to this sequence number have landed and are patched (observed in order,
+                                     // so the parity of a barrier phase never aliases an older one)
+      int qk_next[2] = {0, 1};       // next sequence number whose S the stream issues
+      int pv_next[2] = {0, 1};       // next sequence number whose P V the stream issues
+      PollGuard guard(wl);
+      while (ok && (pv_next[0] < Tall || pv_next[1] < Tall)) {
+        bool progress = false;
+        while (ready + 1 < Tall) {
+          const int slot = (ready + 1) % KV_STAGES, u = (ready + 1) / KV_STAGES;
+          if (!(mbar_test_wait(bar(BT_K_FULL + slot), u & 1) && mbar_test_wait(bar(BT_V_FULL + slot), u & 1) &&
+                mbar_test_wait(bar(BT_PATCHED + slot), u & 1)))
+            break;
           ++ready;
-          const int slot = ready % KV_STAGES, u = ready / KV_STAGES;
-          ok = mbar_wait(bar(BT_K_FULL + slot), u & 1, abort_flag, p.status, wl) &&
-               mbar_wait(bar(BT_V_FULL + slot), u & 1, abort_flag, p.status, wl) &&
-               mbar_wait(bar(BT_PATCHED + slot), u & 1, abort_flag, p.status, wl);
-          tc_fence_after();
+          progress = true;
         }
-      };
-      ok = mbar_wait(bar(BT_Q_FULL), 0, abort_flag, p.status, wl);  // (also when the list is empty: the copy must land)
-#pragma unroll
-      for (int x = 0; x < 2; ++x) {  // prologue: S(x) of the stream's first tile
-        if (T[x] == 0 || !ok) continue;
-        need(x);
-        if (!ok) break;
-        issue_qk(x, x);
-        tc_commit(bar(BT_S_FULL + x));
-        tc_commit(bar(BT_K_EMPTY + x % KV_STAGES));
-      }
-      for (int j = 0; j < T[0] && ok; ++j) {
 #pragma unroll
         for (int x = 0; x < 2; ++x) {
-          if (j >= T[x] || !ok) continue;
-          const int s = 2 * j + x, sn = s + 2;
-          need(s);
-          ok = ok && mbar_wait(bar(BT_P_FULL + x), j & 1, abort_flag, p.status, wl);
-          if (!ok) break;
-          tc_fence_after();
-          issue_pv(x, s, j == 0);
-          tc_commit(bar(BT_O_READY + x));
-          tc_commit(bar(BT_V_EMPTY + s % KV_STAGES));
-          if (j + 1 < T[x]) {
-            need(sn);
-            if (!ok) break;
-            issue_qk(x, sn);
+          if (pv_next[x] < qk_next[x]) {  // S issued: P V as soon as the softmax has written P
+            const int s = pv_next[x], j = s >> 1;
+            if (mbar_test_wait(bar(BT_P_FULL + x), j & 1)) {
+              tc_fence_after();
+              issue_pv(x, s, j == 0);
+              tc_commit(bar(BT_O_READY + x));
+              tc_commit(bar(BT_V_EMPTY + s % KV_STAGES));
+              pv_next[x] = s + 2;
+              progress = true;
+            }
+          }
+          if (qk_next[x] == pv_next[x] && qk_next[x] < Tall && qk_next[x] <= ready) {  // the S buffer is free
+            const int s = qk_next[x];
+            tc_fence_after();
+            issue_qk(x, s);
             tc_commit(bar(BT_S_FULL + x));
-            tc_commit(bar(BT_K_EMPTY + sn % KV_STAGES));
+            tc_commit(bar(BT_K_EMPTY + s % KV_STAGES));
+            qk_next[x] = s + 2;
+            progress = true;
           }
         }
+        if (progress) guard.progress();
+        else ok = guard.idle(abort_flag, p.status);
       }
       if (!ok) {  // make sure no MMA of this thread is still running before TMEM and smem go away
         int dummy = 0;
         tc_commit(bar(BT_DRAIN));
-        mbar_wait(bar(BT_DRAIN), 0, &dummy, nullptr, wl);
+        mbar_wait(bar(BT_DRAIN), 0, &dummy, nullptr);
       }
     }
     __syncwarp();
@@ -376,44 +421,42 @@ branch_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
     // =============================================================== softmax warpgroups (streams)
     const int x = warp >> 2;
     const int row_in_tile = (warp & 3) * 32 + lane;
-    const int R = R0 + row_in_tile;
-    const bool row_valid = R < rows_total;
-    const int tok = R / G, hq = hk * G + R % G;       // token (branch, draft row) and query head of this row
+    const bool row_valid = row_in_tile < rows_here;
+    const int tok = tok0 + row_in_tile / G;          // token (branch, draft row) of this row
     const int rb = tok / n, ri = tok % n;
     const int rj = row_valid ? rb - b_first : -1;    // the row's branch as an index into the tile's branches
     // draft rows of the block this row may see, as bits: its ancestors and itself (a chain: rows 0..i)
     const uint32_t tm = !row_valid ? 0u
                         : (p.tree_mask ? __ldg(p.tree_mask + static_cast<int64_t>(rb) * n + ri) : (2u << ri) - 1u) &
-                              ((n < 32 ? (1u << n) : 0u) - 1u);
+                              ((1u << n) - 1u);
     const uint32_t lane_base = static_cast<uint32_t>((warp & 3) * 32) << 16;
     const uint32_t tS = tmem + lane_base + x * 128;
     const uint32_t tO = tmem + lane_base + 256 + x * 128;
     const float c = p.scale_log2;
     float m_ref = -INFINITY, l = 0.f;
     bool ok = true;
+    int cursor = 0;
     const int Tx = T[x];
     for (int j = 0; j < Tx && ok; ++j) {
       ok = mbar_wait(bar(BT_S_FULL + x), j & 1, abort_flag, p.status, wl);
       if (!ok) break;
       tc_fence_after();
-      // ---- which columns of the tile this row sees
-      const uint32_t e = table[2 * j + x];
-      const int key0 = bt_tile(e) * BT_BN;
+      // ---- which columns of the tile this row sees (a row beyond the tile's rows sees nothing)
+      const BtTile e = tile_at(2 * j + x, cursor);
+      const int key0 = e.tile * BT_BN;
       ColumnBits allow;
-      bool full, any;
-      if (bt_seg(e) == 0xff) {  // shared prefix: every row, up to its end
+      bool full = false;
+      if (e.seg < 0 && row_valid) {  // shared prefix: up to its end
         const int cnt = P - key0;
         full = cnt >= BT_BN;
-        any = true;
 #pragma unroll
         for (int w = 0; w < 4; ++w) {
           const int k = cnt - 32 * w;
           allow.w[w] = k >= 32 ? 0xffffffffu : (k <= 0 ? 0u : (1u << k) - 1u);
         }
-      } else if (bt_seg(e) == rj) {  // the row's own branch: rows before the block, then the block by the mask
+      } else if (e.seg >= 0 && e.seg == rj) {  // the row's own branch: rows before the block, then the block by the mask
         const int hist = len_s[rj] - n - key0;  // column of the block's first row
         full = hist >= BT_BN;
-        any = hist > 0 || tm != 0u;  // (hist + n > 0 always holds for a listed tile)
 #pragma unroll
         for (int w = 0; w < 4; ++w) {
           const int k = hist - 32 * w;
@@ -421,12 +464,10 @@ branch_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
           const uint32_t block = k >= 32 ? 0u : (k >= 0 ? tm << k : (k > -32 ? tm >> (-k) : 0u));
           allow.w[w] = before | block;
         }
-        any = (allow.w[0] | allow.w[1] | allow.w[2] | allow.w[3]) != 0u;
       } else {  // another branch's suffix
-        full = false;
-        any = false;
         allow.w[0] = allow.w[1] = allow.w[2] = allow.w[3] = 0u;
       }
+      const bool any = (allow.w[0] | allow.w[1] | allow.w[2] | allow.w[3]) != 0u;
       auto wait_o = [&] { return mbar_wait(bar(BT_O_READY + x), (j - 1) & 1, abort_flag, p.status, wl); };
       if (__any_sync(0xffffffffu, any)) {
         const bool masked = !__all_sync(0xffffffffu, full);
@@ -446,10 +487,8 @@ branch_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
     }
     pdl_launch_dependents();  // the next kernel of the stream may start its own set-up now
 
-    // ---- merge of the two streams.  Every softmax thread reaches the named barriers below, even one that gave up on
-    // a wait (it only skips its global stores).  (m, l) of a row cross through shared memory -- the K slot of the
-    // stream's last tile, free once its accumulator is complete; a stream without tiles owns slot x, never filled or
-    // long free -- the accumulators are read straight from TMEM: this warpgroup combines columns [64 x, 64 x + 64).
+    // ---- the two streams' (m, l) of a row cross through shared memory: the K slot of the stream's last tile,
+    // free once its accumulator is complete; a stream without tiles owns slot x, never filled or long free
     auto ml_of = [&](int y) {
       const int slot = T[y] > 0 ? (2 * (T[y] - 1) + y) % KV_STAGES : y;
       return reinterpret_cast<float2*>(smem_gen + BT_SMEM_K + slot * BT_TILE_BYTES);
@@ -462,53 +501,37 @@ branch_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
     const float2 oth = ml_of(1 - x)[row_in_tile];
     // a stream whose tiles were all hidden from this row has l = 0 and takes no part
     const float m_own = l > 0.f ? m_ref : -INFINITY, m_oth = oth.y > 0.f ? oth.x : -INFINITY;
-    const float m = fmaxf(m_own, m_oth);
-    const float w_own = l > 0.f ? fast_exp2(m_own - m) : 0.f, w_oth = oth.y > 0.f ? fast_exp2(m_oth - m) : 0.f;
-    const float lsum = l * w_own + oth.y * w_oth;
-    const bool has_own = Tx > 0, has_oth = T[1 - x] > 0;  // a stream without tiles never wrote its accumulator
-    const uint32_t tOwn = tmem + lane_base + 256 + x * 128 + x * 64;
-    const uint32_t tOth = tmem + lane_base + 256 + (1 - x) * 128 + x * 64;
-    const int tid_t = threadIdx.x & 127;
-    // staging for the tiled stores of the output: the Q buffer for warpgroup 0, the first V slot for warpgroup 1
-    // (every MMA and copy of the CTA is complete once both streams have seen their last accumulator)
-    float* stage = reinterpret_cast<float*>(smem_gen + (x == 0 ? BT_SMEM_Q : BT_SMEM_V));
-    const uint32_t stage_addr = smem_base + (x == 0 ? BT_SMEM_Q : BT_SMEM_V);
-    auto store_box = [&](int q2, const float (&v)[32], bool write) {  // columns [64 x + 32 q2, + 32) of all 128 rows
-      stage_box_row(stage + q2 * BT_BOX_FLOATS, row_in_tile, v);
-      fence_proxy_async();
-      asm volatile("bar.sync %0, 128;\n" ::"r"(1 + x) : "memory");
-      if (tid_t == 0 && write) {
-        tma_store_4d(&tm_o, stage_addr + q2 * BT_BOX_FLOATS * 4, x * 64 + q2 * 32, hk * G, R0 / G, 0);
-        tma_store_commit();
-      }
-    };
-    auto store_lse = [&](float mm, float ll) {
-      if (x == 0 && p.lse && row_valid)
-        p.lse[(static_cast<int64_t>(rb) * p.q_heads + hq) * n + ri] = (mm + log2f(ll)) * 0.69314718055994530942f;
-    };
-    if (C == 1) {
-      const float inv = 1.f / lsum;
-      const float a_own = w_own * inv, a_oth = w_oth * inv;
-#pragma unroll
-      for (int q2 = 0; q2 < 2; ++q2) {
-        uint32_t o[32], o2[32];
-        if (has_own) tmem_ld32(tOwn + q2 * 32, o);
-        if (has_oth) tmem_ld32(tOth + q2 * 32, o2);
-        tc_wait_ld();
-        float v[32];
-#pragma unroll
-        for (int i = 0; i < 32; ++i) {
-          v[i] = has_own ? __uint_as_float(o[i]) * a_own : 0.f;
-          if (has_oth) v[i] = fmaf(__uint_as_float(o2[i]), a_oth, v[i]);
-        }
-        store_box(q2, v, ok);
-      }
-      if (tid_t == 0) tma_store_wait_read();
-      if (ok) store_lse(m, lsum);
-    } else {
-      // ---- this CTA's partial -> scratch: [column chunk][row] float4, so a warp writes 512 contiguous bytes
-      float4* gpart = reinterpret_cast<float4*>(p.part + (static_cast<size_t>(unit) * C + crank) * BT_PART_FLOATS);
-      float2* gml = reinterpret_cast<float2*>(p.ml + (static_cast<size_t>(unit) * C + crank) * BT_ML_FLOATS);
+    fin_m = fmaxf(m_own, m_oth);
+    fin_w_own = l > 0.f ? fast_exp2(m_own - fin_m) : 0.f;
+    fin_w_oth = oth.y > 0.f ? fast_exp2(m_oth - fin_m) : 0.f;
+    fin_l = l * fin_w_own + oth.y * fin_w_oth;
+  }
+
+  // ================================================================= merge over the unit's CTAs
+  // Every thread of every CTA of the cluster comes through here, whatever happened above.  Row r of the tile is
+  // finished by CTA r C / 128 (contiguous slices).  Behind the first barrier every MMA and copy of every CTA is
+  // complete and the exchange slots above have been read: the K/V rings are free.
+  auto slice_begin = [&](int d) { return (BT_BM * d + C - 1) / C; };  // first row owned by CTA d
+  const float* recv = reinterpret_cast<const float*>(smem_gen + BT_SMEM_K);  // [source CTA][row of my slice][BT_RECV_STRIDE]
+  const int max_slice = (BT_BM + C - 1) / C;
+  tc_fence_before();
+  if (C > 1) cluster_sync_all();
+  else __syncthreads();
+  tc_fence_after();
+  if (warp < 8) {
+    // ---- push: this thread's row, columns [64 x, 64 x + 64) of both streams combined (unnormalised, relative
+    // to the row's maximum over this CTA's tiles), into the owner's shared memory
+    const int x = warp >> 2, row_in_tile = (warp & 3) * 32 + lane;
+    const bool row_valid = row_in_tile < rows_here;
+    if ((warp & 3) * 32 < rows_here) {  // warp-uniform (the TMEM loads are warp-collective): the warp has a row
+      const int d = min(row_in_tile, rows_here - 1) * C / BT_BM;
+      const uint32_t lane_base = static_cast<uint32_t>((warp & 3) * 32) << 16;
+      const uint32_t tOwn = tmem + lane_base + 256 + x * 128 + x * 64;
+      const uint32_t tOth = tmem + lane_base + 256 + (1 - x) * 128 + x * 64;
+      const bool has_own = T[x] > 0, has_oth = T[1 - x] > 0;  // a stream without tiles never wrote its accumulator
+      const uint32_t local = smem_base + BT_SMEM_K +
+                             ((crank * max_slice + (min(row_in_tile, rows_here - 1) - slice_begin(d))) * BT_RECV_STRIDE) * 4;
+      const uint32_t dst = C > 1 ? cluster_map(local, static_cast<uint32_t>(d)) : local;
 #pragma unroll
       for (int q2 = 0; q2 < 2; ++q2) {
         uint32_t o[32], o2[32];
@@ -520,73 +543,53 @@ branch_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
           float v[4];
 #pragma unroll
           for (int i = 0; i < 4; ++i) {
-            v[i] = has_own ? __uint_as_float(o[4 * cc + i]) * w_own : 0.f;
-            if (has_oth) v[i] = fmaf(__uint_as_float(o2[4 * cc + i]), w_oth, v[i]);
+            v[i] = has_own ? __uint_as_float(o[4 * cc + i]) * fin_w_own : 0.f;
+            if (has_oth) v[i] = fmaf(__uint_as_float(o2[4 * cc + i]), fin_w_oth, v[i]);
           }
-          gpart[(x * 16 + q2 * 8 + cc) * BT_BM + row_in_tile] = make_float4(v[0], v[1], v[2], v[3]);
+          if (row_valid) st_cluster_v4(dst + (x * 64 + q2 * 32 + cc * 4) * 4, v[0], v[1], v[2], v[3]);
         }
       }
-      if (x == 0) gml[row_in_tile] = make_float2(lsum > 0.f ? m : -INFINITY, lsum);
-      // ---- ticket: the partial above must be visible before the ticket is
-      __threadfence();
-      asm volatile("bar.sync 3, 256;\n" ::: "memory");
-      if (threadIdx.x == 0) {
-        int* cnt = p.counters + unit;
-        const bool last = atomicAdd(cnt, 1) == C - 1;
-        if (last) *cnt = 0;  // every CTA of the unit has taken its ticket: ready for the next call
-        __threadfence();     // the others' partials are read after this
-        *last_slot = last ? 1 : 0;
+      if (row_valid && x == 0) st_cluster_v2(dst + BT_D * 4, fin_l > 0.f ? fin_m : -INFINITY, fin_l);
+    }
+  }
+  tc_fence_before();
+  if (C > 1) cluster_sync_all();  // release / acquire over the cluster: every partial has arrived at its owner
+  else __syncthreads();
+  if (warp < 8) {
+    // ---- the owner's rows: (row, 16-byte column chunk) pairs dealt to the 256 threads, the partials added in
+    // CTA order; a warp writes whole 512-byte output rows
+    const bool clean = *abort_flag == 0 && *reinterpret_cast<volatile int*>(p.status) == 0;  // nobody gave up on a wait
+    const int row0 = slice_begin(crank), row1 = min(slice_begin(crank + 1), rows_here);
+    for (int idx = threadIdx.x; idx < (row1 - row0) * 32; idx += 256) {
+      const int ris = idx >> 5, chunk = idx & 31;
+      float M = -INFINITY;
+      for (int cr = 0; cr < C; ++cr) {
+        const float2 ml = *reinterpret_cast<const float2*>(recv + (cr * max_slice + ris) * BT_RECV_STRIDE + BT_D);
+        if (ml.y > 0.f) M = fmaxf(M, ml.x);  // a CTA whose tiles were all hidden from the row has l = 0
       }
-      asm volatile("bar.sync 3, 256;\n" ::: "memory");
-      if (*last_slot) {
-        // ---- the unit's partials in CTA order -> output
-        const bool clean = ok && *reinterpret_cast<volatile int*>(p.status) == 0;  // nobody gave up on a wait
-        const float2* uml = reinterpret_cast<const float2*>(p.ml + static_cast<size_t>(unit) * C * BT_ML_FLOATS);
-        const float4* upart = reinterpret_cast<const float4*>(p.part + static_cast<size_t>(unit) * C * BT_PART_FLOATS);
-        // (weights in registers: the loops over the unit's CTAs are unrolled to their upper bound)
-        float wgt[BT_MAX_CTAS], lcr[BT_MAX_CTAS];
-        float M = -INFINITY;
-#pragma unroll
-        for (int cr = 0; cr < BT_MAX_CTAS; ++cr) {
-          const float2 v = cr < C ? __ldcg(uml + cr * BT_BM + row_in_tile) : make_float2(-INFINITY, 0.f);
-          wgt[cr] = v.y > 0.f ? v.x : -INFINITY;  // a CTA whose tiles were all hidden from the row has l = 0
-          lcr[cr] = v.y;
-          M = fmaxf(M, wgt[cr]);
-        }
-        float lall = 0.f;
-#pragma unroll
-        for (int cr = 0; cr < BT_MAX_CTAS; ++cr) {
-          wgt[cr] = wgt[cr] == -INFINITY ? 0.f : fast_exp2(wgt[cr] - M);
-          lall = fmaf(wgt[cr], lcr[cr], lall);
-        }
+      float lall = 0.f;
+      float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+      for (int cr = 0; cr < C; ++cr) {
+        const float* src = recv + (cr * max_slice + ris) * BT_RECV_STRIDE;
+        const float2 ml = *reinterpret_cast<const float2*>(src + BT_D);
+        const float w = ml.y > 0.f ? fast_exp2(ml.x - M) : 0.f;
+        if (w == 0.f) continue;  // (also a CTA without tiles, whose accumulator was never written)
+        const float4 t = *reinterpret_cast<const float4*>(src + chunk * 4);
+        lall = fmaf(w, ml.y, lall);
+        acc.x = fmaf(w, t.x, acc.x);
+        acc.y = fmaf(w, t.y, acc.y);
+        acc.z = fmaf(w, t.z, acc.z);
+        acc.w = fmaf(w, t.w, acc.w);
+      }
+      if (clean) {
+        const int row = row0 + ris;
+        const int tok = tok0 + row / G, hq = hk * G + row % G;
         const float inv = 1.f / lall;
-#pragma unroll
-        for (int q2 = 0; q2 < 2; ++q2) {
-          float v[32];
-#pragma unroll
-          for (int i = 0; i < 32; ++i) v[i] = 0.f;
-#pragma unroll
-          for (int cr = 0; cr < BT_MAX_CTAS; ++cr) {
-            const float w = wgt[cr];
-            if (cr >= C || w == 0.f) continue;  // (also a CTA without tiles, which wrote no accumulator)
-            const float4* src = upart + static_cast<size_t>(cr) * (BT_PART_FLOATS / 4) + (x * 16 + q2 * 8) * BT_BM + row_in_tile;
-            float4 t[8];
-#pragma unroll
-            for (int cc = 0; cc < 8; ++cc) t[cc] = __ldcg(src + cc * BT_BM);
-#pragma unroll
-            for (int cc = 0; cc < 8; ++cc) {
-              v[4 * cc] = fmaf(w, t[cc].x, v[4 * cc]);
-              v[4 * cc + 1] = fmaf(w, t[cc].y, v[4 * cc + 1]);
-              v[4 * cc + 2] = fmaf(w, t[cc].z, v[4 * cc + 2]);
-              v[4 * cc + 3] = fmaf(w, t[cc].w, v[4 * cc + 3]);
-            }
-          }
-#pragma unroll
-          for (int i = 0; i < 32; ++i) v[i] *= inv;
-          store_box(q2, v, clean);
-        }
-        if (tid_t == 0) tma_store_wait_read();
-        if (clean) store_lse(M, lall);
+        *reinterpret_cast<float4*>(p.out + (static_cast<int64_t>(tok) * p.q_heads + hq) * BT_D + chunk * 4) =
+            make_float4(acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv);
+        if (chunk == 0 && p.lse)
+          p.lse[(static_cast<int64_t>(tok / n) * p.q_heads + hq) * n + tok % n] =
+              (M + log2f(lall)) * 0.69314718055994530942f;
       }
     }
   }
@@ -603,41 +606,111 @@ branch_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
 // ---------------------------------------------------------------- host side
 
 struct BtPlan {
-  int row_tiles, units, ctas_per_unit;
+  int row_tiles, branches_per_tile, slices_per_branch, box_tokens, units, ctas_per_unit;
   bool ok;
 };
 
-static BtPlan bt_plan(int prefix_len, int max_suffix_len, int n_branches, int q_heads, int kv_heads, int q_len,
-                      int sm_count) {
-  BtPlan pl = {0, 0, 1, false};
-  const int G = q_heads / kv_heads, nG = q_len * G;
-  if (G > BT_BM || (G & (G - 1)) != 0) return pl;               // a Q box holds whole tokens: G divides 128
-  if ((BT_BM - 1) / nG + 2 > BT_MAX_BRANCHES) return pl;        // branches with a row in one tile
-  const int64_t rows = static_cast<int64_t>(n_branches) * nG;
-  const int64_t row_tiles = (rows + BT_BM - 1) / BT_BM;
-  const int64_t units = row_tiles * kv_heads;
-  if (units > 65536 / 4) return pl;                              // one counter per unit in the 64 KiB counter block
-  const int64_t Tp = (static_cast<int64_t>(prefix_len) + BT_BN - 1) / BT_BN;
-  if (Tp > 0xffff) return pl;
-  const int nb_max = static_cast<int>(std::min<int64_t>((BT_BM - 1) / nG + 2, n_branches));
-  const int64_t Ts_max = static_cast<int64_t>(nb_max) * ((max_suffix_len + BT_BN - 1) / BT_BN);
-  int c = static_cast<int>(std::max<int64_t>(1, std::min<int64_t>(sm_count / units, BT_MAX_CTAS)));
-  // no more CTAs than pairs of tiles a unit certainly has
-  const int64_t t_min = Tp + (max_suffix_len + BT_BN - 1) / BT_BN;
-  c = static_cast<int>(std::max<int64_t>(1, std::min<int64_t>(c, t_min / 2)));
-  // the tile list of a CTA must fit its table
-  if ((Tp + c - 1) / c + (Ts_max + c - 1) / c + 2 > BT_MAX_TILES) return pl;
-  pl.row_tiles = static_cast<int>(row_tiles);
-  pl.units = static_cast<int>(units);
-  pl.ctas_per_unit = c;
-  pl.ok = true;
-  return pl;
+static cudaError_t bt_set_attributes() {
+  static PerDeviceOnce attr_done;
+  if (attr_done.done()) return cudaSuccess;
+  cudaError_t e = cudaFuncSetAttribute(branch_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, BT_SMEM_BYTES);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(branch_tc_kernel, cudaFuncAttributePreferredSharedMemoryCarveout,
+                             cudaSharedmemCarveoutMaxShared);
+  if (e == cudaSuccess) attr_done.set();
+  return e;
 }
 
-static size_t bt_scratch_bytes(const BtPlan& pl) {
-  if (pl.ctas_per_unit <= 1) return 0;
-  return SCRATCH_COUNTER_BYTES +
-         static_cast<size_t>(pl.units) * pl.ctas_per_unit * (BT_PART_FLOATS + BT_ML_FLOATS) * sizeof(float);
+// How many clusters of c CTAs of the kernel can be resident at once on the current device (0 if the query fails).
+static int bt_resident_clusters(int c) {
+  static std::atomic<int> cache[64][BT_MAX_CTAS + 1];  // per device and cluster size: 0 = not asked yet, else answer + 1
+  int dev = -1;
+  if (c < 1 || c > BT_MAX_CTAS || cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 0;
+  const int cached = cache[dev][c].load(std::memory_order_acquire);
+  if (cached > 0) return cached - 1;
+  int n = 0;
+  if (bt_set_attributes() == cudaSuccess) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(static_cast<unsigned>(c * 64));
+    cfg.blockDim = dim3(BT_THREADS);
+    cfg.dynamicSmemBytes = BT_SMEM_BYTES;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = static_cast<unsigned>(c);
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    int got = 0;
+    if (cudaOccupancyMaxActiveClusters(&got, branch_tc_kernel, &cfg) == cudaSuccess) n = got;
+    else (void)cudaGetLastError();
+  } else {
+    (void)cudaGetLastError();
+  }
+  cache[dev][c].store(n + 1, std::memory_order_release);
+  return n;
+}
+
+// The largest cluster size <= want whose clusters, one per unit, are all resident at once (1 if none is).
+static int bt_cluster_size(int64_t units, int64_t want) {
+  for (int c = static_cast<int>(std::min<int64_t>(want, BT_MAX_CTAS)); c >= 2; --c)
+    if (bt_resident_clusters(c) >= units) return c;
+  return 1;
+}
+
+static BtPlan bt_plan(int prefix_len, int max_suffix_len, int n_branches, int q_heads, int kv_heads, int q_len,
+                      int sm_count) {
+  BtPlan pl = {0, 0, 1, 0, 0, 1, false};
+  const int G = q_heads / kv_heads, nG = q_len * G;
+  const int64_t Tp = (static_cast<int64_t>(prefix_len) + BT_BN - 1) / BT_BN;
+  const int64_t ts_max = (max_suffix_len + BT_BN - 1) / BT_BN;
+  // CTAs per unit for a given number of units: fill the SMs, but no more CTAs than pairs of tiles a unit certainly has
+  auto ctas_for = [&](int64_t units) {
+    const int64_t want = std::min<int64_t>(std::max<int64_t>(sm_count / units, 1), std::max<int64_t>((Tp + ts_max) / 2, 1));
+    return bt_cluster_size(units, want);
+  };
+  if (nG <= BT_BM) {
+    // whole branches per row tile, the same number in every tile.  More, smaller tiles walk the prefix more often
+    // but may fill the machine better: take the tiling with the shortest estimated walk per CTA (a branch's suffix
+    // counted at 0.6 of its longest possible walk).
+    const int per_tile_max = std::min(BT_MAX_BRANCHES, BT_BM / nG);
+    const int tiles_min = (n_branches + per_tile_max - 1) / per_tile_max;
+    const int64_t ts_est = std::max<int64_t>(1, (ts_max * 6 + 9) / 10);
+    int64_t best = -1;
+    for (int tiles = tiles_min; tiles <= std::min(n_branches, 2 * tiles_min); ++tiles) {
+      const int per_tile = (n_branches + tiles - 1) / tiles;
+      if (per_tile > per_tile_max || static_cast<int64_t>(tiles - 1) * per_tile >= n_branches) continue;
+      const int64_t units = static_cast<int64_t>(tiles) * kv_heads;
+      if (units > (1 << 30)) continue;
+      const int c = ctas_for(units);
+      const int64_t waves = (units * c + sm_count - 1) / sm_count;
+      const int64_t est = waves * ((Tp + per_tile * ts_est + c - 1) / c + 3);  // + fixed cost of a CTA, in tiles
+      if (best < 0 || est < best) {
+        best = est;
+        pl.row_tiles = tiles;
+        pl.branches_per_tile = per_tile;
+        pl.box_tokens = per_tile * q_len;
+        pl.units = static_cast<int>(units);
+        pl.ctas_per_unit = c;
+      }
+    }
+    if (best < 0) return pl;
+    pl.slices_per_branch = 1;
+  } else {
+    // a branch has more than 128 rows: 128-row slices, which must start on a token
+    if (BT_BM % G != 0) return pl;
+    pl.slices_per_branch = (nG + BT_BM - 1) / BT_BM;
+    const int64_t tiles = static_cast<int64_t>(n_branches) * pl.slices_per_branch;
+    const int64_t units = tiles * kv_heads;
+    if (units > (1 << 30)) return pl;
+    pl.row_tiles = static_cast<int>(tiles);
+    pl.branches_per_tile = 1;
+    pl.box_tokens = BT_BM / G;
+    pl.units = static_cast<int>(units);
+    pl.ctas_per_unit = ctas_for(units);
+  }
+  pl.ok = true;
+  return pl;
 }
 
 bool branch_tc_supported(const CacheView& suffix, int prefix_len, int max_suffix_len, int n_branches, int q_heads,
@@ -646,34 +719,21 @@ bool branch_tc_supported(const CacheView& suffix, int prefix_len, int max_suffix
   return bt_plan(prefix_len, max_suffix_len, n_branches, q_heads, suffix.kv_heads, q_len, sm_count).ok;
 }
 
-size_t branch_tc_workspace_bytes(int prefix_len, int max_suffix_len, int n_branches, int q_heads, int kv_heads,
-                                 int q_len, int sm_count) {
-  return bt_scratch_bytes(bt_plan(prefix_len, max_suffix_len, n_branches, q_heads, kv_heads, q_len, sm_count));
-}
-
 cudaError_t launch_branch_tc(const bf16* q, const CacheView& prefix, int prefix_len, const CacheView& suffix,
                              const int32_t* d_suffix_len, const uint32_t* d_tree_mask, int max_suffix_len,
                              int n_branches, int q_heads, int q_len, float scale, float* out, float* lse, int* status,
-                             long long wait_limit, void* workspace, size_t workspace_bytes, cudaStream_t st,
-                             LaunchInfo& li, const bf16* k_new, const bf16* v_new) {
-  BtPlan pl = bt_plan(prefix_len, max_suffix_len, n_branches, q_heads, suffix.kv_heads, q_len, li.sm_count);
+                             long long wait_limit, cudaStream_t st, LaunchInfo& li, const bf16* k_new,
+                             const bf16* v_new) {
+  const BtPlan pl = bt_plan(prefix_len, max_suffix_len, n_branches, q_heads, suffix.kv_heads, q_len, li.sm_count);
   if (!pl.ok) return cudaErrorInvalidValue;
-  // several CTAs per unit need the scratch; with too little of it the units are not split
-  while (pl.ctas_per_unit > 1 && (!workspace || bt_scratch_bytes(pl) > workspace_bytes)) pl.ctas_per_unit -= 1;
   const int G = q_heads / suffix.kv_heads;
   const uint64_t tokens = static_cast<uint64_t>(n_branches) * q_len;
-  CUtensorMap tq, tpk, tpv, tsk, tsv, to;
-  {  // q: [tokens][q_heads][128]; a box is [128 / G tokens][G heads][64 columns]: 128 stacked rows in order
+  CUtensorMap tq, tpk, tpv, tsk, tsv;
+  {  // q: [tokens][q_heads][128]; a box is [box_tokens tokens][G heads][64 columns]: the tile's stacked rows in order
     const uint64_t d[4] = {BT_D, static_cast<uint64_t>(q_heads), tokens, 1};
     const uint64_t s[3] = {BT_D * 2ull, static_cast<uint64_t>(q_heads) * BT_D * 2ull, 0};
-    const uint32_t bx[4] = {64, static_cast<uint32_t>(G), static_cast<uint32_t>(BT_BM / G), 1};
+    const uint32_t bx[4] = {64, static_cast<uint32_t>(G), static_cast<uint32_t>(pl.box_tokens), 1};
     if (!make_map_bf16(&tq, q, d, s, bx)) return cudaErrorInvalidValue;
-  }
-  {  // out: same rows, fp32, boxes of 32 columns
-    const uint64_t d[4] = {BT_D, static_cast<uint64_t>(q_heads), tokens, 1};
-    const uint64_t s[3] = {BT_D * 4ull, static_cast<uint64_t>(q_heads) * BT_D * 4ull, 0};
-    const uint32_t bx[4] = {32, static_cast<uint32_t>(G), static_cast<uint32_t>(BT_BM / G), 1};
-    if (!make_map_f32(&to, out, d, s, bx)) return cudaErrorInvalidValue;
   }
   {  // suffix caches: rows at or beyond max_suffix_len read as zero
     const uint64_t d[4] = {BT_D, static_cast<uint64_t>(max_suffix_len), static_cast<uint64_t>(suffix.kv_heads),
@@ -701,6 +761,9 @@ cudaError_t launch_branch_tc(const bf16* q, const CacheView& prefix, int prefix_
   p.prefix_len = prefix_len;
   p.max_suffix_len = max_suffix_len;
   p.row_tiles = pl.row_tiles;
+  p.branches_per_tile = pl.branches_per_tile;
+  p.slices_per_branch = pl.slices_per_branch;
+  p.box_tokens = pl.box_tokens;
   p.ctas_per_unit = pl.ctas_per_unit;
   p.scale_log2 = scale * 1.4426950408889634f;
   p.wait_limit = wait_limit;
@@ -713,24 +776,14 @@ cudaError_t launch_branch_tc(const bf16* q, const CacheView& prefix, int prefix_
   p.sb = suffix.sb;
   p.sh = suffix.sh;
   p.sr = suffix.sr;
+  p.out = out;
   p.lse = lse;
   p.status = status;
-  p.counters = static_cast<int*>(workspace);
-  p.part = pl.ctas_per_unit > 1 ? reinterpret_cast<float*>(static_cast<unsigned char*>(workspace) + SCRATCH_COUNTER_BYTES)
-                                : nullptr;
-  p.ml = pl.ctas_per_unit > 1 ? p.part + static_cast<size_t>(pl.units) * pl.ctas_per_unit * BT_PART_FLOATS : nullptr;
-  static PerDeviceOnce attr_done;
-  if (!attr_done.done()) {
-    cudaError_t e = cudaFuncSetAttribute(branch_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, BT_SMEM_BYTES);
-    if (e == cudaSuccess)
-      e = cudaFuncSetAttribute(branch_tc_kernel, cudaFuncAttributePreferredSharedMemoryCarveout,
-                               cudaSharedmemCarveoutMaxShared);
-    if (e != cudaSuccess) return e;
-    attr_done.set();
-  }
+  cudaError_t e = bt_set_attributes();
+  if (e != cudaSuccess) return e;
   li.launches += 1;
-  return launch_pdl(branch_tc_kernel, dim3(static_cast<unsigned>(pl.units * pl.ctas_per_unit)), dim3(BT_THREADS),
-                    BT_SMEM_BYTES, st, tq, tpk, tpv, tsk, tsv, to, p);
+  return launch_pdl_cluster(branch_tc_kernel, dim3(static_cast<unsigned>(pl.units) * pl.ctas_per_unit), dim3(BT_THREADS),
+                            BT_SMEM_BYTES, st, static_cast<unsigned>(pl.ctas_per_unit), tq, tpk, tpv, tsk, tsv, p);
 }
 
 }  // namespace jup

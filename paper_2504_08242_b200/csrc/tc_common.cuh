@@ -61,6 +61,30 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
   return false;
 }
 
+// For a thread that polls several barriers without blocking on any one of them: call progress() after a pass
+// that found work and idle() after one that did not.  idle() returns false when no pass has found work for
+// limit_cycles SM clocks (the status word is then set), when another thread of the CTA has given up, or when any
+// CTA of this context has.
+struct PollGuard {
+  long long t0, limit;
+  uint32_t it;
+  __device__ __forceinline__ explicit PollGuard(long long limit_cycles) : t0(0), limit(limit_cycles), it(0) {}
+  __device__ __forceinline__ void progress() { it = 0; }
+  __device__ __forceinline__ bool idle(volatile int* abort_flag, int* status) {
+    if (it == 0) t0 = clock64();
+    if ((++it & 127u) != 0u) return true;
+    if (*abort_flag) return false;
+    if (status && *reinterpret_cast<volatile int*>(status) != 0) {
+      *abort_flag = 1;
+      return false;
+    }
+    if (clock64() - t0 <= limit) return true;
+    *abort_flag = 1;
+    if (status) atomicExch(status, 1);
+    return false;
+  }
+};
+
 // ---------------------------------------------------------------- thread-block cluster, distributed shared memory
 __device__ __forceinline__ uint32_t cluster_ctarank() {
   uint32_t r;

@@ -186,10 +186,20 @@ def test_branch_argument_errors(ctx):
         with pytest.raises(J.JupiterError) as e:
             ctx.branch_attn(**a)
         assert e.value.status == status, over
+    # only the split-KV kernel keeps partial results in the context's scratch: a context with too little of it
+    # refuses that kernel and still serves the shapes that the streaming kernel takes
     small = J.Context(0, workspace_bytes=1024)
+    small.select_branch_kernel(J.BRANCH_SPLIT_KV)
     with pytest.raises(J.JupiterError) as e:
         small.branch_attn(q, pd, 32, sd, dl, 20, 3, 4, 2, 0.125, out)
     assert e.value.status == J.ERR_WORKSPACE
+    torch.cuda.synchronize()
+    assert bool((out == 7.0).all())
+    small.select_branch_kernel(J.BRANCH_AUTO)
+    small.branch_attn(q, pd, 32, sd, dl, 20, 3, 4, 2, 0.125, out)
+    torch.cuda.synchronize()
+    assert bool(torch.isfinite(out).all()) and not bool((out == 7.0).all())
+    out.fill_(7.0)
     small.close()
     torch.cuda.synchronize()
     assert bool((out == 7.0).all())

@@ -21,16 +21,6 @@ def ctx():
     c.close()
 
 
-@pytest.fixture(scope="module")
-def ctx_one_cta():
-    """A context whose scratch only holds the counters: every unit is walked by a single CTA."""
-    import paper_2504_08242_b200 as J
-    c = J.Context(0, workspace_bytes=65536 + 4096)
-    c.select_branch_kernel(J.BRANCH_TENSOR_CORE)
-    yield c
-    c.close()
-
-
 def random_tree_masks(seed, B, n):
     picks = synth.uniform_ints(seed, 5, B * n, 0, 1 << 20).reshape(B, n)
     tm = np.zeros((B, n), np.uint32)
@@ -119,9 +109,22 @@ def test_branch_tc_tree(ctx, B, Hq, Hkv, P, n, lens):
 
 
 @pytest.mark.parametrize("mode", ["plain", "fused", "tree"])
-def test_one_cta_per_unit(ctx_one_cta, mode):
-    """Without scratch for partials a unit is walked by one CTA, which writes the output itself."""
-    run_case(ctx_one_cta, 460, 7, 8, 2, 300, 5, [5, 127, 128, 129, 255, 256, 257], mode)
+def test_one_cta_per_unit(ctx, mode):
+    """More (kv head, row tile) units than half the SMs: every unit is walked by a single CTA (no cluster)."""
+    lens = [5 + (37 * i) % 300 for i in range(30)]
+    run_case(ctx, 460, 30, 64, 16, 300, 5, lens, mode)
+
+
+def test_a_branch_larger_than_a_row_tile(ctx):
+    """q_len x group = 256 stacked rows per branch: two 128-row slices of one branch per kv head, the first of
+    which writes the block into the cache."""
+    for mode in ("plain", "fused", "tree"):
+        run_case(ctx, 465, 3, 32, 2, 200, 16, [16, 150, 300], mode)
+
+
+def test_group_sizes_that_are_not_powers_of_two(ctx):
+    run_case(ctx, 466, 5, 6, 2, 130, 4, [4, 60, 129, 200, 7], "fused")      # group 3: 12 rows per branch
+    run_case(ctx, 467, 4, 10, 2, 260, 3, [3, 128, 131, 40], "tree")         # group 5
 
 
 def test_block_straddles_key_tiles(ctx):
@@ -131,9 +134,11 @@ def test_block_straddles_key_tiles(ctx):
         run_case(ctx, 480 + L, 3, 8, 2, 64, 5, [L, L + 1, 5], "tree")
 
 
-def test_long_walk_many_tiles(ctx_one_cta):
-    """One CTA lists more tiles than its rings hold many times over (ring reuse, barrier parities)."""
-    run_case(ctx_one_cta, 490, 4, 8, 2, 3000, 4, [4, 700, 1300, 129], "fused")
+def test_long_walk_many_tiles(ctx):
+    """Every CTA lists more tiles than its rings hold many times over (ring reuse, barrier parities)."""
+    run_case(ctx, 490, 4, 8, 2, 9000, 4, [4, 2500, 4100, 129], "fused")
+    lens = [5 + (41 * i) % 900 for i in range(30)]
+    run_case(ctx, 491, 30, 64, 16, 1500, 5, lens, "fused")  # single-CTA units
 
 
 def test_repeatable_and_matches_the_other_kernels(ctx):
@@ -171,8 +176,7 @@ def test_unsupported_shapes_are_refused_when_pinned(ctx):
     z = lambda *s: torch.zeros(*s, dtype=torch.bfloat16, device="cuda")
     dl = torch.full((2,), 4, dtype=torch.int32, device="cuda")
     for Hq, Hkv, D, n in [(4, 2, 64, 4),      # head_dim 64
-                          (6, 2, 128, 4),     # group of 3
-                          (2, 2, 128, 4)]:    # q_len * group = 4 rows per branch
+                          (34, 2, 128, 16)]:  # 272 rows per branch and a group of 17, which does not divide 128
         pd = J.cache_desc(z(1, Hkv, 32, D), z(1, Hkv, 32, D))
         sd = J.cache_desc(z(2, Hkv, 40, D), z(2, Hkv, 40, D))
         out = torch.zeros(2, n, Hq, D, device="cuda")
