@@ -300,7 +300,7 @@ static jupiter_status branch_attn_impl(jupiter_ctx* ctx, const void* q, const ju
   if (max_suffix_len < q_len || max_suffix_len > sfx.capacity) return JUPITER_ERR_OUT_OF_RANGE;
   if (!aligned16(q) || !aligned16(out)) return JUPITER_ERR_ALIGNMENT;
   // which kernel: few stacked rows per kv head stream through clusters (no scratch); many rows with head_dim 128 go
-  // to the tensor-core kernel (no scratch either); the rest to the split-KV kernel, the only one that can find the
+  // to the tensor-core kernel (which adapts to the scratch it is given); the rest to the split-KV kernel, the only one that can find the
   // scratch too small
   DeviceGuard guard(ctx->device);
   const bool tc_ok = jup::branch_tc_supported(sfx, prefix_len, max_suffix_len, n_branches, q_heads, q_len, scale,
@@ -331,8 +331,8 @@ static jupiter_status branch_attn_impl(jupiter_ctx* ctx, const void* q, const ju
   else if (use_tc)
     e = jup::launch_branch_tc(static_cast<const bf16*>(q), pfx, prefix_len, sfx, d_suffix_len, d_tree_mask,
                               max_suffix_len, n_branches, q_heads, q_len, scale, out, lse, ctx->d_status,
-                              ctx->wait_limit, static_cast<cudaStream_t>(stream), li, static_cast<const bf16*>(k_new),
-                              static_cast<const bf16*>(v_new));
+                              ctx->wait_limit, ctx->workspace, ctx->workspace_bytes, static_cast<cudaStream_t>(stream),
+                              li, static_cast<const bf16*>(k_new), static_cast<const bf16*>(v_new));
   else
     e = jup::launch_branch(static_cast<const bf16*>(q), pfx, prefix_len, sfx, d_suffix_len, d_tree_mask,
                            max_suffix_len, n_branches, q_heads, q_len, scale, out, lse, ctx->workspace,

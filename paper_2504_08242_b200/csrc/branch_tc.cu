@@ -16,20 +16,21 @@
 // so its first loads are in flight while the lengths arrive).  Inside a CTA:
 //   loader warp  : TMA (tiled, 128-byte swizzle) Q once -- one box [tokens][G heads][64] lands in stacked-row
 //                  order -- then the K/V tiles of the CTA's list into 3-stage rings, K and V refilled independently
-//   patch warp   : the last tiles of a branch's suffix hold rows that TMA cannot know about: rows at or beyond the
-//                  device-side length (dead; their V rows are zeroed so that 0 x NaN never reaches an accumulator)
-//                  and, with the fused KVCache write, the rows of this step's block, which are read from
-//                  k_new / v_new into the tile (and stored into the cache by the unit that owns them)
+//   patch warps  : (one for K, one for V) the last tiles of a branch's suffix hold rows that TMA cannot know about:
+//                  rows at or beyond the device-side length (dead; their V rows are zeroed so that 0 x NaN never
+//                  reaches an accumulator) and, with the fused KVCache write, the rows of this step's block, which are
+//                  read from k_new / v_new into the tile (and stored into the cache by the unit that owns them)
 //   MMA warp     : one thread issues tcgen05.mma  S = Q K^T  and  O += P V, accumulators in TMEM; it polls both
 //                  streams and the rings and never blocks on one of them
 //   softmax WGs  : two warpgroups run two independent online-softmax streams over the even and the odd tiles of
 //                  the CTA's list (one thread per row); a warp none of whose rows sees a tile only zeroes its P
 // TMEM (512 columns): S_0 | S_1 | O_0 | O_1.
-// At the end the two streams of a CTA are merged in registers and every row's unnormalised (O, m, l) is pushed
-// into the shared memory of the CTA of the cluster that owns the row (distributed shared memory; the K/V rings are
-// free by then: one cluster barrier before the push says so, a second one after it says that every partial has
-// arrived).  The owner adds the partials in CTA order -- the result never depends on timing -- normalises and
-// writes the output rows.  No global scratch, no atomics, one launch.
+// At the end the two streams of a CTA are merged in registers.  With one CTA per unit the rows are normalised
+// and written out.  Otherwise every CTA writes its rows' unnormalised (O, m, l) to scratch (L2), and behind ONE
+// cluster barrier CTA r of the cluster finishes a contiguous slice of the rows: it adds the partials in CTA
+// order -- the result never depends on timing -- normalises and writes the output.  (Pushing the partials into the
+// owner's shared memory instead was measured: 64 KB per CTA took 2.3 us over distributed shared memory, twice the
+// trip through L2.)  No atomics, no second launch, nothing waits on a flag.
 // All mbarrier waits are bounded; on expiry the CTA sets the status word, drains its own copies and MMAs,
 // frees TMEM and returns (every thread still passes the cluster barriers).
 #include <algorithm>
@@ -51,7 +52,9 @@ constexpr int BT_PANEL_BYTES = 16384;  // 128 rows x 64 elements
 constexpr int BT_KV_STAGES = 3;
 constexpr int BT_MAX_BRANCHES = 32;    // branches in one row tile
 constexpr int BT_MAX_CTAS = 8;         // CTAs per unit (the portable cluster size)
-constexpr int BT_RECV_STRIDE = BT_D + 4;  // floats per received row: O, then (m, l), padded against bank conflicts
+constexpr int BT_RECV_STRIDE = BT_D + 4;  // one CTA per unit: floats per staged row: O, then (m, l), padded against bank conflicts
+constexpr int BT_PART_FLOATS = BT_BM * BT_D;  // one CTA's partial accumulator
+constexpr int BT_ML_FLOATS = BT_BM * 2;       // and its (m, l) pairs
 
 struct BtParams {
   int n_branches, q_len, q_heads, group, kv_heads;
@@ -73,6 +76,8 @@ struct BtParams {
   float* out;
   float* lse;
   int* status;
+  float* part;  // ctas_per_unit > 1: [units][ctas_per_unit][32 column chunks][128 rows] float4, a CTA's partial accumulator
+  float* ml;    //                    [units][ctas_per_unit][128 rows] (m, l)
 };
 
 // shared memory: [Q][K ring][V ring][barriers, flags][lengths and tile counts of the row tile's branches]
@@ -83,11 +88,10 @@ constexpr int BT_SMEM_BAR = BT_SMEM_V + BT_KV_STAGES * BT_TILE_BYTES;
 constexpr int BT_SMEM_LEN = BT_SMEM_BAR + 256;
 constexpr int BT_SMEM_BYTES = BT_SMEM_LEN + 2 * BT_MAX_BRANCHES * 4 + 1024;  // + slack for 1024-byte alignment
 static_assert(BT_SMEM_BYTES <= 227 * 1024, "shared memory per CTA");
-// partials received from the cluster live in the K/V rings: [source CTA][row of the slice][BT_RECV_STRIDE]
-static_assert((BT_BM + BT_MAX_CTAS) * BT_RECV_STRIDE * 4 <= 2 * BT_KV_STAGES * BT_TILE_BYTES, "partials fit in the rings");
+static_assert(BT_BM * BT_RECV_STRIDE * 4 <= 2 * BT_KV_STAGES * BT_TILE_BYTES, "the staged rows fit in the rings");
 constexpr int BT_LOADER_WARP = 8,  // warps 0..7: the two softmax warpgroups
-              BT_MMA_WARP = 9, BT_PATCH_WARP = 10;
-constexpr int BT_THREADS = 32 * 11;
+              BT_MMA_WARP = 9, BT_KPATCH_WARP = 10, BT_VPATCH_WARP = 11;
+constexpr int BT_THREADS = 32 * 12;
 
 enum {
   BT_Q_FULL = 0,
@@ -95,12 +99,13 @@ enum {
   BT_K_EMPTY = 4,   // [3]
   BT_V_FULL = 7,    // [3]
   BT_V_EMPTY = 10,  // [3]
-  BT_PATCHED = 13,  // [3] the patch warp is done with the slot's tile
-  BT_S_FULL = 16,   // [2]
-  BT_P_FULL = 18,   // [2]
-  BT_O_READY = 20,  // [2]
-  BT_DRAIN = 22,
-  BT_BAR_COUNT = 23
+  BT_K_PATCHED = 13,  // [3] the patch warp is done with the K tile of the slot
+  BT_V_PATCHED = 16,  // [3] ... with the V tile
+  BT_S_FULL = 19,     // [2]
+  BT_P_FULL = 21,     // [2]
+  BT_O_READY = 23,    // [2]
+  BT_DRAIN = 25,
+  BT_BAR_COUNT = 26
 };
 
 // One entry of a CTA's tile list.
@@ -109,13 +114,6 @@ struct BtTile {
   int tile;    // tile number inside the segment
   bool patch;  // the patch warp has work on it
 };
-
-__device__ __forceinline__ void st_cluster_v4(uint32_t addr, float a, float b, float c, float d) {
-  asm volatile("st.shared::cluster.v4.f32 [%0], {%1, %2, %3, %4};\n" ::"r"(addr), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
-}
-__device__ __forceinline__ void st_cluster_v2(uint32_t addr, float a, float b) {
-  asm volatile("st.shared::cluster.v2.f32 [%0], {%1, %2};\n" ::"r"(addr), "f"(a), "f"(b) : "memory");
-}
 
 __global__ void __launch_bounds__(BT_THREADS, 1)
 branch_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_pk,
@@ -289,59 +287,53 @@ branch_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
       }
     }
     __syncwarp();
-  } else if (warp == BT_PATCH_WARP) {
-    // =============================================================== patch warp
+  } else if (warp == BT_KPATCH_WARP || warp == BT_VPATCH_WARP) {
+    // =============================================================== patch warps: one for the K ring, one for V
+    const bool is_v = warp == BT_VPATCH_WARP;
+    const int full0 = is_v ? BT_V_FULL : BT_K_FULL, done0 = is_v ? BT_V_PATCHED : BT_K_PATCHED;
+    const uint32_t ring = is_v ? sV : sK;
+    const bf16* fresh = is_v ? p.v_new : p.k_new;
+    bf16* cache = is_v ? p.v_cache : p.k_cache;
     bool ok = true;
     int cursor = 0;
     for (int s = 0; s < Tall && ok; ++s) {
       const int slot = s % KV_STAGES, u = s / KV_STAGES;
-      // one lane spins; the others then observe the completed phases themselves (a single test each)
-      if (lane == 0)
-        ok = mbar_wait(bar(BT_K_FULL + slot), u & 1, abort_flag, p.status, wl) &&
-             mbar_wait(bar(BT_V_FULL + slot), u & 1, abort_flag, p.status, wl);
+      // one lane spins; the others then observe the completed phase themselves (a single test each)
+      if (lane == 0) ok = mbar_wait(bar(full0 + slot), u & 1, abort_flag, p.status, wl);
       ok = __shfl_sync(0xffffffffu, ok, 0);
-      if (!ok) break;
-      if (lane != 0)
-        ok = mbar_wait(bar(BT_K_FULL + slot), u & 1, abort_flag, p.status, wl) &&
-             mbar_wait(bar(BT_V_FULL + slot), u & 1, abort_flag, p.status, wl);
+      if (ok && lane != 0) ok = mbar_wait(bar(full0 + slot), u & 1, abort_flag, p.status, wl);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       const BtTile e = tile_at(s, cursor);
-      if (e.patch) {
-        const int j = e.seg, b = b_first + j, L = len_s[j], key0 = e.tile * BT_BN;
+      // K: the rows of this step's block (dead rows need nothing: their scores are masked).  V: the block's rows,
+      // and zeros in the dead rows so that 0 x NaN never reaches the accumulator.
+      if (e.patch && (is_v || fused)) {
+        const int b = b_first + e.seg, L = len_s[e.seg], key0 = e.tile * BT_BN;
         const int new_begin = fused ? L - n : L;
         const int r_begin = max(new_begin - key0, 0);
+        const int r_end = is_v ? BT_BN : min(L - key0, BT_BN);
         // the block's rows go into the cache once per (branch, kv head): by the unit whose row tile starts the branch
         const bool writer = fused && (p.slices_per_branch == 1 || rt % p.slices_per_branch == 0);
-        const uint32_t kslot = sK + slot * BT_TILE_BYTES, vslot = sV + slot * BT_TILE_BYTES;
-        for (int idx = lane; idx < (BT_BN - r_begin) * 16; idx += 32) {
-          const int r = r_begin + (idx >> 4), c = idx & 15;
-          const int key = key0 + r;
+        const uint32_t tile_addr = ring + slot * BT_TILE_BYTES;
+        for (int idx = lane; idx < (r_end - r_begin) * 16; idx += 32) {
+          const int r = r_begin + (idx >> 4), c = idx & 15, key = key0 + r;
           // 16-byte piece c of row r in the 128-byte-swizzled two-panel tile
-          const uint32_t off = (c >> 3) * BT_PANEL_BYTES + r * 128 + (((c & 7) ^ (r & 7)) << 4);
-          if (key < L) {  // a row of this step's block
-            const int64_t src = ((static_cast<int64_t>(b) * n + (key - new_begin)) * p.kv_heads + hk) * BT_D + c * 8;
-            const uint4 kk = __ldg(reinterpret_cast<const uint4*>(p.k_new + src));
-            const uint4 vv = __ldg(reinterpret_cast<const uint4*>(p.v_new + src));
-            asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};\n" ::"r"(kslot + off), "r"(kk.x), "r"(kk.y), "r"(kk.z),
-                         "r"(kk.w)
+          const uint32_t dst = tile_addr + (c >> 3) * BT_PANEL_BYTES + r * 128 + (((c & 7) ^ (r & 7)) << 4);
+          if (key < L) {
+            const uint4 w = __ldg(reinterpret_cast<const uint4*>(
+                fresh + ((static_cast<int64_t>(b) * n + (key - new_begin)) * p.kv_heads + hk) * BT_D + c * 8));
+            asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};\n" ::"r"(dst), "r"(w.x), "r"(w.y), "r"(w.z), "r"(w.w)
                          : "memory");
-            asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};\n" ::"r"(vslot + off), "r"(vv.x), "r"(vv.y), "r"(vv.z),
-                         "r"(vv.w)
-                         : "memory");
-            if (writer) {
-              const int64_t dst = b * p.sb + hk * p.sh + static_cast<int64_t>(key) * p.sr + c * 8;
-              *reinterpret_cast<uint4*>(p.k_cache + dst) = kk;
-              *reinterpret_cast<uint4*>(p.v_cache + dst) = vv;
-            }
-          } else {  // a dead row: its scores are masked, its V row must not poison the accumulator
-            asm volatile("st.shared.v4.u32 [%0], {%1, %1, %1, %1};\n" ::"r"(vslot + off), "r"(0u) : "memory");
+            if (writer)
+              *reinterpret_cast<uint4*>(cache + b * p.sb + hk * p.sh + static_cast<int64_t>(key) * p.sr + c * 8) = w;
+          } else {
+            asm volatile("st.shared.v4.u32 [%0], {%1, %1, %1, %1};\n" ::"r"(dst), "r"(0u) : "memory");
           }
         }
         fence_proxy_async();  // the tensor cores read the slot through the async proxy
       }
       __syncwarp();
-      if (lane == 0) mbar_arrive(bar(BT_PATCHED + slot));
+      if (lane == 0) mbar_arrive(bar(done0 + slot));
     }
   } else if (warp == BT_MMA_WARP) {
     // =============================================================== MMA issuer
@@ -369,26 +361,30 @@ branch_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
       // both streams' P, and issues whatever is ready.  Per stream the order is fixed: S(s) -> [softmax] -> P V(s)
       // -> S(s + 2), because the stream has one S buffer.
       bool ok = mbar_wait(bar(BT_Q_FULL), 0, abort_flag, p.status, wl);  // (also when the list is empty: the copy must land)
-      int ready = -1;                // tiles up to this sequence number have landed and are patched (observed in order,
-                                     // so the parity of a barrier phase never aliases an older one)
+      int k_ready = -1, v_ready = -1;  // K / V tiles up to this sequence number have landed and are patched (observed
+                                       // in order, so the parity of a barrier phase never aliases an older one)
       int qk_next[2] = {0, 1};       // next sequence number whose S the stream issues
       int pv_next[2] = {0, 1};       // next sequence number whose P V the stream issues
       PollGuard guard(wl);
       while (ok && (pv_next[0] < Tall || pv_next[1] < Tall)) {
         bool progress = false;
-        while (ready + 1 < Tall) {
-          const int slot = (ready + 1) % KV_STAGES, u = (ready + 1) / KV_STAGES;
-          if (!(mbar_test_wait(bar(BT_K_FULL + slot), u & 1) && mbar_test_wait(bar(BT_V_FULL + slot), u & 1) &&
-                mbar_test_wait(bar(BT_PATCHED + slot), u & 1)))
-            break;
-          ++ready;
+        while (k_ready + 1 < Tall) {
+          const int slot = (k_ready + 1) % KV_STAGES, u = (k_ready + 1) / KV_STAGES;
+          if (!(mbar_test_wait(bar(BT_K_FULL + slot), u & 1) && mbar_test_wait(bar(BT_K_PATCHED + slot), u & 1))) break;
+          ++k_ready;
+          progress = true;
+        }
+        while (v_ready + 1 < Tall) {
+          const int slot = (v_ready + 1) % KV_STAGES, u = (v_ready + 1) / KV_STAGES;
+          if (!(mbar_test_wait(bar(BT_V_FULL + slot), u & 1) && mbar_test_wait(bar(BT_V_PATCHED + slot), u & 1))) break;
+          ++v_ready;
           progress = true;
         }
 #pragma unroll
         for (int x = 0; x < 2; ++x) {
           if (pv_next[x] < qk_next[x]) {  // S issued: P V as soon as the softmax has written P
             const int s = pv_next[x], j = s >> 1;
-            if (mbar_test_wait(bar(BT_P_FULL + x), j & 1)) {
+            if (s <= v_ready && mbar_test_wait(bar(BT_P_FULL + x), j & 1)) {
               tc_fence_after();
               issue_pv(x, s, j == 0);
               tc_commit(bar(BT_O_READY + x));
@@ -397,7 +393,7 @@ branch_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
               progress = true;
             }
           }
-          if (qk_next[x] == pv_next[x] && qk_next[x] < Tall && qk_next[x] <= ready) {  // the S buffer is free
+          if (qk_next[x] == pv_next[x] && qk_next[x] < Tall && qk_next[x] <= k_ready) {  // the S buffer is free
             const int s = qk_next[x];
             tc_fence_after();
             issue_qk(x, s);
@@ -505,33 +501,134 @@ branch_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
     fin_w_own = l > 0.f ? fast_exp2(m_own - fin_m) : 0.f;
     fin_w_oth = oth.y > 0.f ? fast_exp2(m_oth - fin_m) : 0.f;
     fin_l = l * fin_w_own + oth.y * fin_w_oth;
+    if (C > 1) {
+      // ---- this CTA's partial of the row -> scratch, as [column chunk][row] float4 so that a warp writes 512
+      // contiguous bytes: columns [64 x, 64 x + 64) of both streams combined, unnormalised, relative to the row's
+      // maximum over this CTA's tiles
+      float4* gpart = reinterpret_cast<float4*>(p.part + (static_cast<size_t>(unit) * C + crank) * BT_PART_FLOATS);
+      float2* gml = reinterpret_cast<float2*>(p.ml + (static_cast<size_t>(unit) * C + crank) * BT_ML_FLOATS);
+      const bool has_own = Tx > 0, has_oth = T[1 - x] > 0;  // a stream without tiles never wrote its accumulator
+      if ((warp & 3) * 32 < rows_here) {  // warp-uniform (the TMEM loads are warp-collective): the warp has a row
+        const uint32_t tOwn = tmem + lane_base + 256 + x * 128 + x * 64;
+        const uint32_t tOth = tmem + lane_base + 256 + (1 - x) * 128 + x * 64;
+#pragma unroll
+        for (int q2 = 0; q2 < 2; ++q2) {
+          uint32_t o[32], o2[32];
+          if (has_own) tmem_ld32(tOwn + q2 * 32, o);
+          if (has_oth) tmem_ld32(tOth + q2 * 32, o2);
+          tc_wait_ld();
+#pragma unroll
+          for (int cc = 0; cc < 8; ++cc) {
+            float v[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              v[i] = has_own ? __uint_as_float(o[4 * cc + i]) * fin_w_own : 0.f;
+              if (has_oth) v[i] = fmaf(__uint_as_float(o2[4 * cc + i]), fin_w_oth, v[i]);
+            }
+            if (row_valid) gpart[(x * 16 + q2 * 8 + cc) * BT_BM + row_in_tile] = make_float4(v[0], v[1], v[2], v[3]);
+          }
+        }
+        if (row_valid && x == 0) gml[row_in_tile] = make_float2(fin_l > 0.f ? fin_m : -INFINITY, fin_l);
+      }
+      __threadfence();  // visible to the cluster before its barrier is passed
+    }
   }
 
-  // ================================================================= merge over the unit's CTAs
-  // Every thread of every CTA of the cluster comes through here, whatever happened above.  Row r of the tile is
-  // finished by CTA r C / 128 (contiguous slices).  Behind the first barrier every MMA and copy of every CTA is
-  // complete and the exchange slots above have been read: the K/V rings are free.
-  auto slice_begin = [&](int d) { return (BT_BM * d + C - 1) / C; };  // first row owned by CTA d
-  const float* recv = reinterpret_cast<const float*>(smem_gen + BT_SMEM_K);  // [source CTA][row of my slice][BT_RECV_STRIDE]
-  const int max_slice = (BT_BM + C - 1) / C;
-  tc_fence_before();
-  if (C > 1) cluster_sync_all();
-  else __syncthreads();
-  tc_fence_after();
-  if (warp < 8) {
-    // ---- push: this thread's row, columns [64 x, 64 x + 64) of both streams combined (unnormalised, relative
-    // to the row's maximum over this CTA's tiles), into the owner's shared memory
-    const int x = warp >> 2, row_in_tile = (warp & 3) * 32 + lane;
-    const bool row_valid = row_in_tile < rows_here;
-    if ((warp & 3) * 32 < rows_here) {  // warp-uniform (the TMEM loads are warp-collective): the warp has a row
-      const int d = min(row_in_tile, rows_here - 1) * C / BT_BM;
+  // ================================================================= output
+  // Every thread of every CTA comes through here, whatever happened above.
+  auto slice_begin = [&](int d) { return (BT_BM * d + C - 1) / C; };  // first row finished by CTA d of the cluster
+  if (C > 1) {
+    // ---- several CTAs per unit: behind the cluster barrier every CTA's partial is in the scratch (L2).  This CTA
+    // finishes the rows [128 crank / C, 128 (crank + 1) / C).  First the normalised weight of every (CTA, row)
+    // into shared memory, then (row, 16-byte column chunk) pairs dealt to the 256 threads with the row running
+    // fastest (a warp reads contiguous pieces of every partial; a pair's loads are issued together, two pairs at a
+    // time); the sums run in CTA order, so the result never depends on timing.
+    tc_fence_before();
+    cluster_sync_all();
+    if (warp < 8) {
+      const bool clean = *abort_flag == 0 && *reinterpret_cast<volatile int*>(p.status) == 0;  // nobody gave up on a wait
+      const float2* uml = reinterpret_cast<const float2*>(p.ml + static_cast<size_t>(unit) * C * BT_ML_FLOATS);
+      const float4* upart = reinterpret_cast<const float4*>(p.part + static_cast<size_t>(unit) * C * BT_PART_FLOATS);
+      float* wtab = reinterpret_cast<float*>(smem_gen + BT_SMEM_K);  // [CTA][row of my slice] (the rings are free)
+      const int row0 = slice_begin(crank), nrows = min(slice_begin(crank + 1), rows_here) - row0;
+      const int max_slice = (BT_BM + C - 1) / C;
+      if (static_cast<int>(threadIdx.x) < nrows) {
+        const int row = row0 + threadIdx.x;
+        float2 ml[BT_MAX_CTAS];
+#pragma unroll
+        for (int cr = 0; cr < BT_MAX_CTAS; ++cr)
+          ml[cr] = cr < C ? __ldcg(uml + cr * BT_BM + row) : make_float2(-INFINITY, 0.f);
+        float M = -INFINITY;
+#pragma unroll
+        for (int cr = 0; cr < BT_MAX_CTAS; ++cr)
+          if (ml[cr].y > 0.f) M = fmaxf(M, ml[cr].x);  // a CTA whose tiles were all hidden from the row has l = 0
+        float w[BT_MAX_CTAS], lall = 0.f;
+#pragma unroll
+        for (int cr = 0; cr < BT_MAX_CTAS; ++cr) {
+          w[cr] = ml[cr].y > 0.f ? fast_exp2(ml[cr].x - M) : 0.f;
+          lall = fmaf(w[cr], ml[cr].y, lall);
+        }
+        const float inv = 1.f / lall;
+#pragma unroll
+        for (int cr = 0; cr < BT_MAX_CTAS; ++cr)
+          if (cr < C) wtab[cr * max_slice + threadIdx.x] = w[cr] * inv;
+        if (clean && p.lse) {
+          const int tok = tok0 + row / G, hq = hk * G + row % G;
+          p.lse[(static_cast<int64_t>(tok / n) * p.q_heads + hq) * n + tok % n] = (M + log2f(lall)) * 0.69314718055994530942f;
+        }
+      }
+      asm volatile("bar.sync 3, 256;\n" ::: "memory");
+      const int pairs = nrows * 32;
+      for (int idx0 = threadIdx.x; idx0 < pairs; idx0 += 512) {
+        float4 t[2][BT_MAX_CTAS];
+        int ris[2], chunk[2];
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          const int idx = min(idx0 + h * 256, pairs - 1);
+          ris[h] = idx % nrows;
+          chunk[h] = idx / nrows;
+#pragma unroll
+          for (int cr = 0; cr < BT_MAX_CTAS; ++cr)
+            if (cr < C)
+              t[h][cr] = __ldcg(upart + static_cast<size_t>(cr) * (BT_PART_FLOATS / 4) + chunk[h] * BT_BM + row0 + ris[h]);
+        }
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+          for (int cr = 0; cr < BT_MAX_CTAS; ++cr) {
+            if (cr >= C) continue;
+            const float w = wtab[cr * max_slice + ris[h]];
+            if (w == 0.f) continue;  // (also a CTA without tiles, whose partial holds nothing meaningful)
+            acc.x = fmaf(w, t[h][cr].x, acc.x);
+            acc.y = fmaf(w, t[h][cr].y, acc.y);
+            acc.z = fmaf(w, t[h][cr].z, acc.z);
+            acc.w = fmaf(w, t[h][cr].w, acc.w);
+          }
+          if (clean && idx0 + h * 256 < pairs) {
+            const int row = row0 + ris[h];
+            const int tok = tok0 + row / G, hq = hk * G + row % G;
+            *reinterpret_cast<float4*>(p.out + (static_cast<int64_t>(tok) * p.q_heads + hq) * BT_D + chunk[h] * 4) = acc;
+          }
+        }
+      }
+    }
+  } else {
+    // ---- one CTA per unit: the rows are staged in shared memory (every MMA and copy of the CTA is complete behind
+    // the barrier, so the K/V rings are free) and written out as whole 512-byte rows
+    float* stage = reinterpret_cast<float*>(smem_gen + BT_SMEM_K);  // [row][BT_RECV_STRIDE]
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    if (warp < 8 && (warp & 3) * 32 < rows_here) {  // warp-uniform (the TMEM loads are warp-collective)
+      const int x = warp >> 2, row_in_tile = (warp & 3) * 32 + lane;
       const uint32_t lane_base = static_cast<uint32_t>((warp & 3) * 32) << 16;
       const uint32_t tOwn = tmem + lane_base + 256 + x * 128 + x * 64;
       const uint32_t tOth = tmem + lane_base + 256 + (1 - x) * 128 + x * 64;
       const bool has_own = T[x] > 0, has_oth = T[1 - x] > 0;  // a stream without tiles never wrote its accumulator
-      const uint32_t local = smem_base + BT_SMEM_K +
-                             ((crank * max_slice + (min(row_in_tile, rows_here - 1) - slice_begin(d))) * BT_RECV_STRIDE) * 4;
-      const uint32_t dst = C > 1 ? cluster_map(local, static_cast<uint32_t>(d)) : local;
+      const float inv = 1.f / fin_l;
+      const float a_own = fin_w_own * inv, a_oth = fin_w_oth * inv;
+      float* dst = stage + row_in_tile * BT_RECV_STRIDE + x * 64;
 #pragma unroll
       for (int q2 = 0; q2 < 2; ++q2) {
         uint32_t o[32], o2[32];
@@ -543,53 +640,27 @@ branch_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
           float v[4];
 #pragma unroll
           for (int i = 0; i < 4; ++i) {
-            v[i] = has_own ? __uint_as_float(o[4 * cc + i]) * fin_w_own : 0.f;
-            if (has_oth) v[i] = fmaf(__uint_as_float(o2[4 * cc + i]), fin_w_oth, v[i]);
+            v[i] = has_own ? __uint_as_float(o[4 * cc + i]) * a_own : 0.f;
+            if (has_oth) v[i] = fmaf(__uint_as_float(o2[4 * cc + i]), a_oth, v[i]);
           }
-          if (row_valid) st_cluster_v4(dst + (x * 64 + q2 * 32 + cc * 4) * 4, v[0], v[1], v[2], v[3]);
+          *reinterpret_cast<float4*>(dst + q2 * 32 + cc * 4) = make_float4(v[0], v[1], v[2], v[3]);
         }
       }
-      if (row_valid && x == 0) st_cluster_v2(dst + BT_D * 4, fin_l > 0.f ? fin_m : -INFINITY, fin_l);
+      if (x == 0) *reinterpret_cast<float2*>(stage + row_in_tile * BT_RECV_STRIDE + BT_D) = make_float2(fin_m, fin_l);
     }
-  }
-  tc_fence_before();
-  if (C > 1) cluster_sync_all();  // release / acquire over the cluster: every partial has arrived at its owner
-  else __syncthreads();
-  if (warp < 8) {
-    // ---- the owner's rows: (row, 16-byte column chunk) pairs dealt to the 256 threads, the partials added in
-    // CTA order; a warp writes whole 512-byte output rows
-    const bool clean = *abort_flag == 0 && *reinterpret_cast<volatile int*>(p.status) == 0;  // nobody gave up on a wait
-    const int row0 = slice_begin(crank), row1 = min(slice_begin(crank + 1), rows_here);
-    for (int idx = threadIdx.x; idx < (row1 - row0) * 32; idx += 256) {
-      const int ris = idx >> 5, chunk = idx & 31;
-      float M = -INFINITY;
-      for (int cr = 0; cr < C; ++cr) {
-        const float2 ml = *reinterpret_cast<const float2*>(recv + (cr * max_slice + ris) * BT_RECV_STRIDE + BT_D);
-        if (ml.y > 0.f) M = fmaxf(M, ml.x);  // a CTA whose tiles were all hidden from the row has l = 0
-      }
-      float lall = 0.f;
-      float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-      for (int cr = 0; cr < C; ++cr) {
-        const float* src = recv + (cr * max_slice + ris) * BT_RECV_STRIDE;
-        const float2 ml = *reinterpret_cast<const float2*>(src + BT_D);
-        const float w = ml.y > 0.f ? fast_exp2(ml.x - M) : 0.f;
-        if (w == 0.f) continue;  // (also a CTA without tiles, whose accumulator was never written)
-        const float4 t = *reinterpret_cast<const float4*>(src + chunk * 4);
-        lall = fmaf(w, ml.y, lall);
-        acc.x = fmaf(w, t.x, acc.x);
-        acc.y = fmaf(w, t.y, acc.y);
-        acc.z = fmaf(w, t.z, acc.z);
-        acc.w = fmaf(w, t.w, acc.w);
-      }
-      if (clean) {
-        const int row = row0 + ris;
+    __syncthreads();
+    if (warp < 8) {
+      const bool clean = *abort_flag == 0 && *reinterpret_cast<volatile int*>(p.status) == 0;  // nobody gave up on a wait
+      for (int idx = threadIdx.x; idx < rows_here * 32 && clean; idx += 256) {
+        const int row = idx >> 5, chunk = idx & 31;
         const int tok = tok0 + row / G, hq = hk * G + row % G;
-        const float inv = 1.f / lall;
         *reinterpret_cast<float4*>(p.out + (static_cast<int64_t>(tok) * p.q_heads + hq) * BT_D + chunk * 4) =
-            make_float4(acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv);
-        if (chunk == 0 && p.lse)
+            *reinterpret_cast<const float4*>(stage + row * BT_RECV_STRIDE + chunk * 4);
+        if (chunk == 0 && p.lse) {
+          const float2 ml = *reinterpret_cast<const float2*>(stage + row * BT_RECV_STRIDE + BT_D);
           p.lse[(static_cast<int64_t>(tok / n) * p.q_heads + hq) * n + tok % n] =
-              (M + log2f(lall)) * 0.69314718055994530942f;
+              (ml.x + log2f(ml.y)) * 0.69314718055994530942f;
+        }
       }
     }
   }
@@ -713,6 +784,17 @@ static BtPlan bt_plan(int prefix_len, int max_suffix_len, int n_branches, int q_
   return pl;
 }
 
+static size_t bt_scratch_bytes(const BtPlan& pl) {
+  if (pl.ctas_per_unit <= 1) return 0;
+  return SCRATCH_COUNTER_BYTES +
+         static_cast<size_t>(pl.units) * pl.ctas_per_unit * (BT_PART_FLOATS + BT_ML_FLOATS) * sizeof(float);
+}
+
+size_t branch_tc_workspace_bytes(int prefix_len, int max_suffix_len, int n_branches, int q_heads, int kv_heads,
+                                 int q_len, int sm_count) {
+  return bt_scratch_bytes(bt_plan(prefix_len, max_suffix_len, n_branches, q_heads, kv_heads, q_len, sm_count));
+}
+
 bool branch_tc_supported(const CacheView& suffix, int prefix_len, int max_suffix_len, int n_branches, int q_heads,
                          int q_len, float scale, int sm_count) {
   if (suffix.head_dim != BT_D || !(scale > 0.f) || !(scale < INFINITY) || encode_fn() == nullptr) return false;
@@ -722,10 +804,12 @@ bool branch_tc_supported(const CacheView& suffix, int prefix_len, int max_suffix
 cudaError_t launch_branch_tc(const bf16* q, const CacheView& prefix, int prefix_len, const CacheView& suffix,
                              const int32_t* d_suffix_len, const uint32_t* d_tree_mask, int max_suffix_len,
                              int n_branches, int q_heads, int q_len, float scale, float* out, float* lse, int* status,
-                             long long wait_limit, cudaStream_t st, LaunchInfo& li, const bf16* k_new,
-                             const bf16* v_new) {
-  const BtPlan pl = bt_plan(prefix_len, max_suffix_len, n_branches, q_heads, suffix.kv_heads, q_len, li.sm_count);
+                             long long wait_limit, void* workspace, size_t workspace_bytes, cudaStream_t st,
+                             LaunchInfo& li, const bf16* k_new, const bf16* v_new) {
+  BtPlan pl = bt_plan(prefix_len, max_suffix_len, n_branches, q_heads, suffix.kv_heads, q_len, li.sm_count);
   if (!pl.ok) return cudaErrorInvalidValue;
+  // several CTAs per unit exchange partials through the scratch; without enough of it a unit is walked by one CTA
+  if (pl.ctas_per_unit > 1 && (!workspace || bt_scratch_bytes(pl) > workspace_bytes)) pl.ctas_per_unit = 1;
   const int G = q_heads / suffix.kv_heads;
   const uint64_t tokens = static_cast<uint64_t>(n_branches) * q_len;
   CUtensorMap tq, tpk, tpv, tsk, tsv;
@@ -779,6 +863,9 @@ cudaError_t launch_branch_tc(const bf16* q, const CacheView& prefix, int prefix_
   p.out = out;
   p.lse = lse;
   p.status = status;
+  p.part = pl.ctas_per_unit > 1 ? reinterpret_cast<float*>(static_cast<unsigned char*>(workspace) + SCRATCH_COUNTER_BYTES)
+                                : nullptr;
+  p.ml = pl.ctas_per_unit > 1 ? p.part + static_cast<size_t>(pl.units) * pl.ctas_per_unit * BT_PART_FLOATS : nullptr;
   cudaError_t e = bt_set_attributes();
   if (e != cudaSuccess) return e;
   li.launches += 1;

@@ -101,14 +101,15 @@ cudaError_t launch_branch_stream(const bf16* q, const CacheView& prefix, int pre
 // Branch attention on tcgen05 / TMEM for many stacked rows per kv head (head_dim 128, positive finite scale; a
 // branch's q_len x group rows must fit a 128-row tile or the group size must divide 128): units of (kv head, row
 // tile) walk prefix + suffixes with one softmax state per row; the CTAs that share a unit form a thread-block
-// cluster and merge through distributed shared memory.  No scratch.  Both calls need the target device current.
+// cluster and exchange their partials through the scratch (with too little of it a unit is walked by one CTA, so
+// the call never fails for lack of scratch).  Both calls need the target device current.
 bool branch_tc_supported(const CacheView& suffix, int prefix_len, int max_suffix_len, int n_branches, int q_heads,
                          int q_len, float scale, int sm_count);
 cudaError_t launch_branch_tc(const bf16* q, const CacheView& prefix, int prefix_len, const CacheView& suffix,
                              const int32_t* d_suffix_len, const uint32_t* d_tree_mask, int max_suffix_len,
                              int n_branches, int q_heads, int q_len, float scale, float* out, float* lse, int* status,
-                             long long wait_limit, cudaStream_t st, LaunchInfo& li, const bf16* k_new = nullptr,
-                             const bf16* v_new = nullptr);
+                             long long wait_limit, void* workspace, size_t workspace_bytes, cudaStream_t st,
+                             LaunchInfo& li, const bf16* k_new = nullptr, const bf16* v_new = nullptr);
 
 // One CTA that waits, for at most limit_cycles SM clocks, on a barrier nobody arrives at, then reports through the
 // status word like any kernel whose bounded wait ran out.
