@@ -16,12 +16,12 @@
 // so its first loads are in flight while the lengths arrive).  Inside a CTA:
 //   loader warp  : TMA (tiled, 128-byte swizzle) Q once -- one box [tokens][G heads][64] lands in stacked-row
 //                  order -- then the K/V tiles of the CTA's list into 3-stage rings, K and V refilled independently
-//   patch warps  : (one for K, one for V) the last tiles of a branch's suffix hold rows that TMA cannot know about:
-//                  rows at or beyond the device-side length (dead; their V rows are zeroed so that 0 x NaN never
-//                  reaches an accumulator) and, with the fused KVCache write, the rows of this step's block, which are
-//                  read from k_new / v_new into the tile (and stored into the cache by the unit that owns them)
-//   MMA warp     : one thread issues tcgen05.mma  S = Q K^T  and  O += P V, accumulators in TMEM; it polls both
-//                  streams and the rings and never blocks on one of them
+//   patch warp   : passes landed tiles on to the MMA issuers, after patching those that need it: the last tiles of a
+//                  branch's suffix hold rows that TMA cannot know about: rows at or beyond the device-side length
+//                  (dead; their V rows are zeroed so that 0 x NaN never reaches an accumulator) and, with the fused
+//                  KVCache write, the rows of this step's block, which are read from k_new / v_new into the tile
+//                  (and stored into the cache by the unit that owns them)
+//   MMA warps    : one thread per stream issues its tcgen05.mma  S = Q K^T  and  O += P V, accumulators in TMEM
 //   softmax WGs  : two warpgroups run two independent online-softmax streams over the even and the odd tiles of
 //                  the CTA's list (one thread per row); a warp none of whose rows sees a tile only zeroes its P
 // TMEM (512 columns): S_0 | S_1 | O_0 | O_1.
@@ -90,7 +90,8 @@ constexpr int BT_SMEM_BYTES = BT_SMEM_LEN + 2 * BT_MAX_BRANCHES * 4 + 1024;  // 
 static_assert(BT_SMEM_BYTES <= 227 * 1024, "shared memory per CTA");
 static_assert(BT_BM * BT_RECV_STRIDE * 4 <= 2 * BT_KV_STAGES * BT_TILE_BYTES, "the staged rows fit in the rings");
 constexpr int BT_LOADER_WARP = 8,  // warps 0..7: the two softmax warpgroups
-              BT_MMA_WARP = 9, BT_KPATCH_WARP = 10, BT_VPATCH_WARP = 11;
+              BT_MMA_WARP = 9,  // and 10: one issuer per stream
+              BT_PATCH_WARP = 11;
 constexpr int BT_THREADS = 32 * 12;
 
 enum {
@@ -99,13 +100,11 @@ enum {
   BT_K_EMPTY = 4,   // [3]
   BT_V_FULL = 7,    // [3]
   BT_V_EMPTY = 10,  // [3]
-  BT_K_PATCHED = 13,  // [3] the patch warp is done with the K tile of the slot
-  BT_V_PATCHED = 16,  // [3] ... with the V tile
-  BT_S_FULL = 19,     // [2]
-  BT_P_FULL = 21,     // [2]
-  BT_O_READY = 23,    // [2]
-  BT_DRAIN = 25,
-  BT_BAR_COUNT = 26
+  BT_S_FULL = 13,   // [2]
+  BT_P_FULL = 15,   // [2]
+  BT_O_READY = 17,  // [2]
+  BT_DRAIN = 19,    // [2]
+  BT_BAR_COUNT = 21
 };
 
 // One entry of a CTA's tile list.
@@ -128,6 +127,8 @@ branch_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
   volatile int* abort_flag = reinterpret_cast<volatile int*>(smem_gen + BT_SMEM_BAR + 8 * BT_BAR_COUNT);
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem_gen + BT_SMEM_BAR + 8 * BT_BAR_COUNT + 8);
   volatile int* suffix_share = reinterpret_cast<volatile int*>(smem_gen + BT_SMEM_BAR + 8 * BT_BAR_COUNT + 16);  // [2]
+  // how many K / V tiles of the list are ready for the tensor cores (landed and patched), published by the loader warp
+  const uint32_t k_ready = sBar + 8 * BT_BAR_COUNT + 24, v_ready = k_ready + 4;
   int* len_s = reinterpret_cast<int*>(smem_gen + BT_SMEM_LEN);  // clamped suffix length of the tile's branches
   int* cum_s = len_s + BT_MAX_BRANCHES;                         // one past the last suffix tile of each
   auto bar = [&](int i) { return sBar + 8u * i; };
@@ -163,6 +164,8 @@ branch_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
   if (threadIdx.x == 0) {
     for (int i = 0; i < BT_BAR_COUNT; ++i) mbar_init(bar(i), (i == BT_P_FULL || i == BT_P_FULL + 1) ? 128u : 1u);
     *abort_flag = 0;
+    count_publish(k_ready, 0);
+    count_publish(v_ready, 0);
     mbar_fence_init();
   }
   if (warp == BT_MMA_WARP) {
@@ -287,129 +290,144 @@ branch_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
       }
     }
     __syncwarp();
-  } else if (warp == BT_KPATCH_WARP || warp == BT_VPATCH_WARP) {
-    // =============================================================== patch warps: one for the K ring, one for V
-    const bool is_v = warp == BT_VPATCH_WARP;
-    const int full0 = is_v ? BT_V_FULL : BT_K_FULL, done0 = is_v ? BT_V_PATCHED : BT_K_PATCHED;
-    const uint32_t ring = is_v ? sV : sK;
-    const bf16* fresh = is_v ? p.v_new : p.k_new;
-    bf16* cache = is_v ? p.v_cache : p.k_cache;
-    bool ok = true;
-    int cursor = 0;
-    for (int s = 0; s < Tall && ok; ++s) {
+  } else if (warp == BT_PATCH_WARP) {
+    // =============================================================== patcher
+    // One warp-uniform event loop: lane 0 watches the K and the V tiles land (each ring in list order); a landed
+    // tile is patched by the whole warp where it needs it and then passed on to the MMA issuers by publishing
+    // the ring's count of ready tiles.
+    // Patching.  K: the rows of this step's block come from k_new (dead rows need nothing: their scores are
+    // masked).  V: the block's rows from v_new, and zeros in the dead rows so that 0 x NaN never reaches the
+    // accumulator.  The block's rows go into the cache once per (branch, kv head): by the unit whose row tile
+    // starts the branch.
+    const bool writer = fused && (p.slices_per_branch == 1 || rt % p.slices_per_branch == 0);
+    auto pass_on = [&](bool is_v, int s, int& cursor) {
       const int slot = s % KV_STAGES, u = s / KV_STAGES;
-      // one lane spins; the others then observe the completed phase themselves (a single test each)
-      if (lane == 0) ok = mbar_wait(bar(full0 + slot), u & 1, abort_flag, p.status, wl);
-      ok = __shfl_sync(0xffffffffu, ok, 0);
-      if (ok && lane != 0) ok = mbar_wait(bar(full0 + slot), u & 1, abort_flag, p.status, wl);
-      ok = __all_sync(0xffffffffu, ok);
-      if (!ok) break;
       const BtTile e = tile_at(s, cursor);
-      // K: the rows of this step's block (dead rows need nothing: their scores are masked).  V: the block's rows,
-      // and zeros in the dead rows so that 0 x NaN never reaches the accumulator.
+      bool landed = true;  // (lane 0 has seen the tile land)
       if (e.patch && (is_v || fused)) {
+        // the other lanes observe the completed phase themselves before they touch the tile
+        landed = lane == 0 || mbar_wait(bar((is_v ? BT_V_FULL : BT_K_FULL) + slot), u & 1, abort_flag, p.status, wl);
+        landed = __all_sync(0xffffffffu, landed);
+      }
+      if (landed && e.patch && (is_v || fused)) {
         const int b = b_first + e.seg, L = len_s[e.seg], key0 = e.tile * BT_BN;
         const int new_begin = fused ? L - n : L;
-        const int r_begin = max(new_begin - key0, 0);
-        const int r_end = is_v ? BT_BN : min(L - key0, BT_BN);
-        // the block's rows go into the cache once per (branch, kv head): by the unit whose row tile starts the branch
-        const bool writer = fused && (p.slices_per_branch == 1 || rt % p.slices_per_branch == 0);
-        const uint32_t tile_addr = ring + slot * BT_TILE_BYTES;
-        for (int idx = lane; idx < (r_end - r_begin) * 16; idx += 32) {
-          const int r = r_begin + (idx >> 4), c = idx & 15, key = key0 + r;
-          // 16-byte piece c of row r in the 128-byte-swizzled two-panel tile
-          const uint32_t dst = tile_addr + (c >> 3) * BT_PANEL_BYTES + r * 128 + (((c & 7) ^ (r & 7)) << 4);
-          if (key < L) {
-            const uint4 w = __ldg(reinterpret_cast<const uint4*>(
-                fresh + ((static_cast<int64_t>(b) * n + (key - new_begin)) * p.kv_heads + hk) * BT_D + c * 8));
-            asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};\n" ::"r"(dst), "r"(w.x), "r"(w.y), "r"(w.z), "r"(w.w)
+        const int r_begin = max(new_begin - key0, 0);     // first row that is new or dead
+        const int r_new = min(L - key0, BT_BN);           // rows [r_begin, r_new) are the block's, the rest is dead
+        const bf16* fresh = is_v ? p.v_new : p.k_new;
+        bf16* cache = is_v ? p.v_cache : p.k_cache;
+        const uint32_t tile_addr = (is_v ? sV : sK) + slot * BT_TILE_BYTES;
+        // 16-byte piece c of row r in the 128-byte-swizzled two-panel tile
+        auto piece = [&](int r, int c) { return tile_addr + (c >> 3) * BT_PANEL_BYTES + r * 128 + (((c & 7) ^ (r & 7)) << 4); };
+        // the block's rows: at most 16 rows x 16 pieces = 8 per lane, all loads in flight at once
+        uint4 w[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+          const int idx = lane + 32 * k, r = r_begin + (idx >> 4), c = idx & 15;
+          if (r < r_new)
+            w[k] = __ldg(reinterpret_cast<const uint4*>(
+                fresh + ((static_cast<int64_t>(b) * n + (key0 + r - new_begin)) * p.kv_heads + hk) * BT_D + c * 8));
+        }
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+          const int idx = lane + 32 * k, r = r_begin + (idx >> 4), c = idx & 15;
+          if (r < r_new) {
+            asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};\n" ::"r"(piece(r, c)), "r"(w[k].x), "r"(w[k].y),
+                         "r"(w[k].z), "r"(w[k].w)
                          : "memory");
             if (writer)
-              *reinterpret_cast<uint4*>(cache + b * p.sb + hk * p.sh + static_cast<int64_t>(key) * p.sr + c * 8) = w;
-          } else {
-            asm volatile("st.shared.v4.u32 [%0], {%1, %1, %1, %1};\n" ::"r"(dst), "r"(0u) : "memory");
+              *reinterpret_cast<uint4*>(cache + b * p.sb + hk * p.sh + static_cast<int64_t>(key0 + r) * p.sr + c * 8) = w[k];
           }
         }
+        if (is_v)
+          for (int idx = lane; idx < (BT_BN - max(r_new, 0)) * 16; idx += 32)
+            asm volatile("st.shared.v4.u32 [%0], {%1, %1, %1, %1};\n" ::"r"(piece(max(r_new, 0) + (idx >> 4), idx & 15)), "r"(0u)
+                         : "memory");
         fence_proxy_async();  // the tensor cores read the slot through the async proxy
       }
       __syncwarp();
-      if (lane == 0) mbar_arrive(bar(done0 + slot));
+      if (lane == 0 && landed) count_publish(is_v ? v_ready : k_ready, s + 1);
+      return landed;
+    };
+    bool ok = true;
+    int kp = 0, vp = 0, kp_cursor = 0, vp_cursor = 0;  // next tiles to pass on
+    PollGuard guard(wl);
+    while (ok && (kp < Tall || vp < Tall)) {
+      int ev = 0;  // 1: K tile kp has landed; 2: V tile vp has landed
+      if (lane == 0) {
+        if (kp < Tall && mbar_test_wait(bar(BT_K_FULL + kp % KV_STAGES), (kp / KV_STAGES) & 1)) ev |= 1;
+        if (vp < Tall && mbar_test_wait(bar(BT_V_FULL + vp % KV_STAGES), (vp / KV_STAGES) & 1)) ev |= 2;
+      }
+      ev = __shfl_sync(0xffffffffu, ev, 0);
+      if (ev & 1) ok = pass_on(false, kp++, kp_cursor) && ok;
+      if (ev & 2) ok = pass_on(true, vp++, vp_cursor) && ok;
+      if (ev) guard.progress();
+      else ok = guard.idle(abort_flag, p.status);
+      ok = __shfl_sync(0xffffffffu, ok, 0);
     }
-  } else if (warp == BT_MMA_WARP) {
-    // =============================================================== MMA issuer
+  } else if (warp == BT_MMA_WARP || warp == BT_MMA_WARP + 1) {
+    // =============================================================== MMA issuers, one thread per stream
+    // Stream x's order is fixed -- S(s) -> [softmax] -> P V(s) -> S(s + 2), the stream has one S buffer -- so its
+    // issuer simply blocks on what comes next; the two streams never wait for each other.
     if (lane == 0) {
+      const int x = warp - BT_MMA_WARP;
       constexpr uint32_t idesc_qk = tc_idesc_bf16(BT_BM, BT_BN, false, false);
       constexpr uint32_t idesc_pv = tc_idesc_bf16(BT_BM, BT_D, false, true);
-      auto s_col = [&](int x) { return tmem + x * 128; };
-      auto o_col = [&](int x) { return tmem + 256 + x * 128; };
-      auto issue_qk = [&](int x, int s) {  // S(x) = Q K^T, K of sequence number s
+      const uint32_t s_col = tmem + x * 128, o_col = tmem + 256 + x * 128;
+      auto issue_qk = [&](int s) {  // S = Q K^T, K of sequence number s
         const uint32_t kb = sK + (s % KV_STAGES) * BT_TILE_BYTES;
 #pragma unroll
         for (int ks = 0; ks < BT_D / 16; ++ks) {
           const uint32_t off = (ks >> 2) * BT_PANEL_BYTES + (ks & 3) * 32;
-          tc_mma_ss(s_col(x), tc_smem_desc(sQ + off, 16, 1024), tc_smem_desc(kb + off, 16, 1024), idesc_qk, ks > 0);
+          tc_mma_ss(s_col, tc_smem_desc(sQ + off, 16, 1024), tc_smem_desc(kb + off, 16, 1024), idesc_qk, ks > 0);
         }
       };
-      auto issue_pv = [&](int x, int s, bool first) {  // O(x) (+)= P(x) V, V of sequence number s
+      auto issue_pv = [&](int s, bool first) {  // O (+)= P V, V of sequence number s
         const uint32_t vb = sV + (s % KV_STAGES) * BT_TILE_BYTES;
 #pragma unroll
         for (int ks = 0; ks < BT_BN / 16; ++ks)
-          tc_mma_ts(o_col(x), s_col(x) + ks * 8, tc_smem_desc(vb + ks * 2048, BT_PANEL_BYTES, 1024), idesc_pv,
+          tc_mma_ts(o_col, s_col + ks * 8, tc_smem_desc(vb + ks * 2048, BT_PANEL_BYTES, 1024), idesc_pv,
                     (!first || ks > 0));
       };
-      // The issuer never blocks on one stream while the other has work: each pass looks at what has landed and at
-      // both streams' P, and issues whatever is ready.  Per stream the order is fixed: S(s) -> [softmax] -> P V(s)
-      // -> S(s + 2), because the stream has one S buffer.
       bool ok = mbar_wait(bar(BT_Q_FULL), 0, abort_flag, p.status, wl);  // (also when the list is empty: the copy must land)
-      int k_ready = -1, v_ready = -1;  // K / V tiles up to this sequence number have landed and are patched (observed
-                                       // in order, so the parity of a barrier phase never aliases an older one)
-      int qk_next[2] = {0, 1};       // next sequence number whose S the stream issues
-      int pv_next[2] = {0, 1};       // next sequence number whose P V the stream issues
-      PollGuard guard(wl);
-      while (ok && (pv_next[0] < Tall || pv_next[1] < Tall)) {
-        bool progress = false;
-        while (k_ready + 1 < Tall) {
-          const int slot = (k_ready + 1) % KV_STAGES, u = (k_ready + 1) / KV_STAGES;
-          if (!(mbar_test_wait(bar(BT_K_FULL + slot), u & 1) && mbar_test_wait(bar(BT_K_PATCHED + slot), u & 1))) break;
-          ++k_ready;
-          progress = true;
+      auto need_k = [&](int s) {
+        ok = ok && count_wait(k_ready, s + 1, abort_flag, p.status, wl);
+        tc_fence_after();
+      };
+      auto need_v = [&](int s) {
+        ok = ok && count_wait(v_ready, s + 1, abort_flag, p.status, wl);
+        tc_fence_after();
+      };
+      const int Tx = T[x];
+      if (Tx > 0 && ok) {
+        need_k(x);
+        if (ok) {
+          issue_qk(x);
+          tc_commit(bar(BT_S_FULL + x));
+          tc_commit(bar(BT_K_EMPTY + x % KV_STAGES));
         }
-        while (v_ready + 1 < Tall) {
-          const int slot = (v_ready + 1) % KV_STAGES, u = (v_ready + 1) / KV_STAGES;
-          if (!(mbar_test_wait(bar(BT_V_FULL + slot), u & 1) && mbar_test_wait(bar(BT_V_PATCHED + slot), u & 1))) break;
-          ++v_ready;
-          progress = true;
+      }
+      for (int j = 0; j < Tx && ok; ++j) {
+        const int s = 2 * j + x, sn = s + 2;
+        need_v(s);
+        ok = ok && mbar_wait(bar(BT_P_FULL + x), j & 1, abort_flag, p.status, wl);
+        if (!ok) break;
+        tc_fence_after();
+        issue_pv(s, j == 0);
+        tc_commit(bar(BT_O_READY + x));
+        tc_commit(bar(BT_V_EMPTY + s % KV_STAGES));
+        if (j + 1 < Tx) {
+          need_k(sn);
+          if (!ok) break;
+          issue_qk(sn);
+          tc_commit(bar(BT_S_FULL + x));
+          tc_commit(bar(BT_K_EMPTY + sn % KV_STAGES));
         }
-#pragma unroll
-        for (int x = 0; x < 2; ++x) {
-          if (pv_next[x] < qk_next[x]) {  // S issued: P V as soon as the softmax has written P
-            const int s = pv_next[x], j = s >> 1;
-            if (s <= v_ready && mbar_test_wait(bar(BT_P_FULL + x), j & 1)) {
-              tc_fence_after();
-              issue_pv(x, s, j == 0);
-              tc_commit(bar(BT_O_READY + x));
-              tc_commit(bar(BT_V_EMPTY + s % KV_STAGES));
-              pv_next[x] = s + 2;
-              progress = true;
-            }
-          }
-          if (qk_next[x] == pv_next[x] && qk_next[x] < Tall && qk_next[x] <= k_ready) {  // the S buffer is free
-            const int s = qk_next[x];
-            tc_fence_after();
-            issue_qk(x, s);
-            tc_commit(bar(BT_S_FULL + x));
-            tc_commit(bar(BT_K_EMPTY + s % KV_STAGES));
-            qk_next[x] = s + 2;
-            progress = true;
-          }
-        }
-        if (progress) guard.progress();
-        else ok = guard.idle(abort_flag, p.status);
       }
       if (!ok) {  // make sure no MMA of this thread is still running before TMEM and smem go away
         int dummy = 0;
-        tc_commit(bar(BT_DRAIN));
-        mbar_wait(bar(BT_DRAIN), 0, &dummy, nullptr);
+        tc_commit(bar(BT_DRAIN + x));
+        mbar_wait(bar(BT_DRAIN + x), 0, &dummy, nullptr);
       }
     }
     __syncwarp();
@@ -434,10 +452,8 @@ branch_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
     int cursor = 0;
     const int Tx = T[x];
     for (int j = 0; j < Tx && ok; ++j) {
-      ok = mbar_wait(bar(BT_S_FULL + x), j & 1, abort_flag, p.status, wl);
-      if (!ok) break;
-      tc_fence_after();
-      // ---- which columns of the tile this row sees (a row beyond the tile's rows sees nothing)
+      // ---- which columns of the tile this row sees (a row beyond the tile's rows sees nothing); worked out while
+      // the tensor cores still compute the tile's scores
       const BtTile e = tile_at(2 * j + x, cursor);
       const int key0 = e.tile * BT_BN;
       ColumnBits allow;
@@ -463,10 +479,13 @@ branch_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
       } else {  // another branch's suffix
         allow.w[0] = allow.w[1] = allow.w[2] = allow.w[3] = 0u;
       }
-      const bool any = (allow.w[0] | allow.w[1] | allow.w[2] | allow.w[3]) != 0u;
+      const bool warp_sees = __any_sync(0xffffffffu, (allow.w[0] | allow.w[1] | allow.w[2] | allow.w[3]) != 0u);
+      const bool masked = !__all_sync(0xffffffffu, full);
+      ok = mbar_wait(bar(BT_S_FULL + x), j & 1, abort_flag, p.status, wl);
+      if (!ok) break;
+      tc_fence_after();
       auto wait_o = [&] { return mbar_wait(bar(BT_O_READY + x), (j - 1) & 1, abort_flag, p.status, wl); };
-      if (__any_sync(0xffffffffu, any)) {
-        const bool masked = !__all_sync(0xffffffffu, full);
+      if (warp_sees) {
         ok = softmax_tile_step<true>(tS, tO, j, masked, allow, c, m_ref, l, wait_o);
       } else {  // no row of this warp sees the tile: P = 0, nothing else changes
         uint32_t z[16];

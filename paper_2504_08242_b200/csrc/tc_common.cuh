@@ -34,6 +34,22 @@ __device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
+// Test that may suspend the thread for a short, hardware-chosen time while the phase is incomplete: a loop around
+// it polls far less often than one around the non-blocking test, which leaves issue slots and shared-memory
+// bandwidth to the warps that compute.
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n"
+      ".reg .pred p;\n"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+      "selp.b32 %0, 1, 0, p;\n"
+      "}\n"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
 
 // Bounded wait (about a second of SM clocks).  Returns false when the limit is hit, when another
 // thread of the CTA has already given up (abort flag in shared memory) or when any CTA of this
@@ -46,8 +62,40 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
   if (mbar_test_wait(bar, parity)) return true;
   const long long t0 = clock64();
   for (uint32_t it = 1;; ++it) {
-    if (mbar_test_wait(bar, parity)) return true;
-    if ((it & 127u) == 0u) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((it & 15u) == 0u) {
+      if (*abort_flag) return false;
+      if (status && *reinterpret_cast<volatile int*>(status) != 0) {
+        *abort_flag = 1;
+        return false;
+      }
+      if (clock64() - t0 > limit_cycles) break;
+    }
+  }
+  *abort_flag = 1;
+  if (status) atomicExch(status, 1);
+  return false;
+}
+
+// A counter in shared memory that one thread advances (release) and others wait on (acquire), for hand-offs that
+// several threads observe: unlike a barrier phase, a count cannot be mistaken for an older one.
+__device__ __forceinline__ void count_publish(uint32_t addr, int value) {
+  asm volatile("st.release.cta.shared::cta.b32 [%0], %1;\n" ::"r"(addr), "r"(value) : "memory");
+}
+__device__ __forceinline__ int count_read(uint32_t addr) {
+  int v;
+  asm volatile("ld.acquire.cta.shared::cta.b32 %0, [%1];\n" : "=r"(v) : "r"(addr) : "memory");
+  return v;
+}
+// Bounded wait until the counter reaches `need`; gives up like mbar_wait.
+__device__ __forceinline__ bool count_wait(uint32_t addr, int need, volatile int* abort_flag, int* status,
+                                           long long limit_cycles) {
+  if (count_read(addr) >= need) return true;
+  const long long t0 = clock64();
+  for (uint32_t it = 1;; ++it) {
+    if (count_read(addr) >= need) return true;
+    __nanosleep(32);  // leave the issue slots to the warps that compute
+    if ((it & 63u) == 0u) {
       if (*abort_flag) return false;
       if (status && *reinterpret_cast<volatile int*>(status) != 0) {
         *abort_flag = 1;
@@ -72,6 +120,7 @@ struct PollGuard {
   __device__ __forceinline__ void progress() { it = 0; }
   __device__ __forceinline__ bool idle(volatile int* abort_flag, int* status) {
     if (it == 0) t0 = clock64();
+    __nanosleep(32);  // leave the issue slots to the warps that compute
     if ((++it & 127u) != 0u) return true;
     if (*abort_flag) return false;
     if (status && *reinterpret_cast<volatile int*>(status) != 0) {
@@ -281,6 +330,14 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32
       : "memory");
 }
 
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];\n"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr)
+      : "memory");
+}
 __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16]) {
   asm volatile(
       "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};\n" ::"r"(

@@ -1,9 +1,11 @@
 // One online-softmax step of the tcgen05 attention kernels: a thread owns one query row (one TMEM lane) and
-// walks the 128 fp32 scores of the current key tile twice with tcgen05.ld -- first the masked row maximum
-// (eight independent chains of 3-input max), then P = exp2(s * c - m) with fp32-pair arithmetic, written back in
-// place as bf16 pairs (P column k holds keys 2k and 2k + 1, so the writes stay behind the reads; the next 32
-// columns are in flight while the current 32 are processed).  The running sum stays in fp32 and the
-// accumulator O is rescaled lazily, only when the row maximum outgrew the reference by more than 2^8.
+// walks the 128 fp32 scores of the current key tile ONCE, in four chunks of 32 columns (tcgen05.ld, the next chunk
+// in flight while the current one is processed): chunk maximum, then P = exp2(s * c - m) with fp32-pair
+// arithmetic, written back in place as bf16 pairs (P column k holds keys 2k and 2k + 1, so the writes stay behind
+// the reads).  The reference maximum m is lazy: it only moves when a chunk's maximum outgrew it by more than 2^8;
+// then the row sum, the P chunks of this tile written so far and -- at the end of the tile -- the accumulator O are
+// scaled by exp2(m_old - m_new).  With well-behaved scores that happens in a row's first chunk and almost never
+// again, so a tile costs one pass over TMEM instead of a maximum pass plus an exponential pass.
 #pragma once
 #include "tc_common.cuh"
 
@@ -21,73 +23,28 @@ struct ColumnBits {  // bit (col & 31) of w[col >> 5] set: visible
   __device__ __forceinline__ bool operator()(int col) const { return (w[col >> 5] >> (col & 31)) & 1u; }
 };
 
+__device__ __forceinline__ uint32_t scale_bf16_pair(uint32_t pair, float a) {
+  const float lo = __uint_as_float(pair << 16), hi = __uint_as_float(pair & 0xffff0000u);
+  return pack_bf16(lo * a, hi * a);
+}
+
 // tS / tO: TMEM addresses (lane base included) of the row's 128 scores and of its 128 accumulator columns.
 // j: number of tiles this stream has processed before (0: O holds nothing yet).
 // masked: warp-uniform; when false every column is visible and `allow` is not consulted.
-// PARTIAL: the stream may meet rows that see none of a tile (their reference maximum stays -inf and P is 0).
+// PARTIAL: the stream may meet rows that see none of a tile (their reference maximum stays -inf and P is 0);
+// otherwise every row sees column 0 of its first tile.
 // wait_o(): waits until O(j-1) is complete (called exactly once when j > 0); returns false if the wait gave up,
 // and then so does this function.  On return P is complete in TMEM (tcgen05.wait::st done); the caller fences
 // and signals the MMA issuer.
 template <bool PARTIAL, class Allow, class WaitO>
 __device__ __forceinline__ bool softmax_tile_step(uint32_t tS, uint32_t tO, int j, bool masked, const Allow& allow,
                                                   float c, float& m_ref, float& l, WaitO&& wait_o) {
-  // ---- pass 1: row maximum
-  float mx;
-  {
-    float a[8];
-#pragma unroll
-    for (int k = 0; k < 8; ++k) a[k] = -INFINITY;
-#pragma unroll
-    for (int h2 = 0; h2 < 2; ++h2) {
-      uint32_t r0[32], r1[32];
-      tmem_ld32(tS + h2 * 64, r0);
-      tmem_ld32(tS + h2 * 64 + 32, r1);
-      tc_wait_ld();
-      if (masked) {
-#pragma unroll
-        for (int i = 0; i < 32; ++i) {
-          if (!allow(h2 * 64 + i)) r0[i] = 0xff800000u;  // -inf
-          if (!allow(h2 * 64 + 32 + i)) r1[i] = 0xff800000u;
-        }
-      }
-#pragma unroll
-      for (int i = 0; i < 32; i += 16)
-#pragma unroll
-        for (int k = 0; k < 8; ++k) {
-          a[k] = fmax3(a[k], __uint_as_float(r0[i + 2 * k]), __uint_as_float(r0[i + 2 * k + 1]));
-          a[k] = fmax3(a[k], __uint_as_float(r1[i + 2 * k]), __uint_as_float(r1[i + 2 * k + 1]));
-        }
-    }
-    mx = fmax3(fmax3(a[0], a[1], a[2]), fmax3(a[3], a[4], a[5]), fmaxf(a[6], a[7]));
-  }
-  const float mxs = mx * c;
-  // lazy rescale: the reference maximum only moves when the true maximum outgrew it by 2^8 (a row that has seen
-  // nothing keeps -inf, and its first visible score moves it because -inf + 8 is still -inf)
-  const bool grow = PARTIAL ? (mxs > m_ref + TC_RESCALE_THRESHOLD) : ((j == 0) || (mxs > m_ref + TC_RESCALE_THRESHOLD));
-  bool o_waited = false;
-  if (j > 0 && __any_sync(0xffffffffu, grow)) {
-    const float alpha = grow ? fast_exp2(m_ref - mxs) : 1.f;
-    l *= alpha;
-    if (!wait_o()) return false;  // O(j-1) must be complete before it is rescaled
-    o_waited = true;
-    tc_fence_after();
-#pragma unroll
-    for (int q4 = 0; q4 < 4; ++q4) {
-      uint32_t o[32];
-      tmem_ld32(tO + q4 * 32, o);
-      tc_wait_ld();
-#pragma unroll
-      for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
-      tmem_st32(tO + q4 * 32, o);
-    }
-  }
-  if (grow) m_ref = mxs;
-  // ---- pass 2: P
-  const float nm = (PARTIAL && m_ref == -INFINITY) ? 0.f : -m_ref;
-  const uint64_t c2 = pack2(c, c), nm2 = pack2(nm, nm);
-  uint64_t lacc[4];
+  const uint64_t c2 = pack2(c, c);
+  uint64_t lacc[4];  // this tile's row sum, four chains
 #pragma unroll
   for (int k = 0; k < 4; ++k) lacc[k] = pack2(0.f, 0.f);
+  float alpha_total = 1.f;  // what the sum and the accumulator of the tiles before this one must be scaled by
+  bool moved = false;       // warp-uniform: some row's reference moved during this tile
   uint32_t sb[2][32];
   tmem_ld32(tS, sb[0]);
 #pragma unroll
@@ -98,8 +55,46 @@ __device__ __forceinline__ bool softmax_tile_step(uint32_t tS, uint32_t tO, int 
     if (masked) {
 #pragma unroll
       for (int i = 0; i < 32; ++i)
-        if (!allow(q4 * 32 + i)) sv[i] = 0xff800000u;
+        if (!allow(q4 * 32 + i)) sv[i] = 0xff800000u;  // -inf
     }
+    // ---- chunk maximum (eight chains of 3-input max)
+    float a[8];
+#pragma unroll
+    for (int k = 0; k < 8; ++k)
+      a[k] = fmax3(__uint_as_float(sv[4 * k]), __uint_as_float(sv[4 * k + 1]), __uint_as_float(sv[4 * k + 2]));
+    const float mx = fmax3(fmax3(fmax3(a[0], a[1], a[2]), fmax3(a[3], a[4], a[5]), fmaxf(a[6], a[7])),
+                           fmax3(__uint_as_float(sv[3]), __uint_as_float(sv[7]), __uint_as_float(sv[11])),
+                           fmax3(fmax3(__uint_as_float(sv[15]), __uint_as_float(sv[19]), __uint_as_float(sv[23])),
+                                 __uint_as_float(sv[27]), __uint_as_float(sv[31])));
+    const float mxs = mx * c;
+    // lazy reference: it only moves when the maximum outgrew it by 2^8 (a row that has seen nothing keeps -inf,
+    // and its first visible score moves it because -inf + 8 is still -inf)
+    const bool grow = mxs > m_ref + TC_RESCALE_THRESHOLD;
+    if (__any_sync(0xffffffffu, grow)) {
+      const float alpha = grow ? fast_exp2(m_ref - mxs) : 1.f;
+      const uint64_t al2 = pack2(alpha, alpha);
+#pragma unroll
+      for (int k = 0; k < 4; ++k) lacc[k] = mul2(lacc[k], al2);
+      if (q4 > 0) {  // the P chunks of this tile written so far were relative to the old reference
+        tc_wait_st();
+#pragma unroll
+        for (int qq = 0; qq < 3; ++qq) {
+          if (qq >= q4) break;
+          uint32_t pk[16];
+          tmem_ld16(tS + qq * 16, pk);
+          tc_wait_ld();  // (also completes the load of the next chunk, which is consumed later anyway)
+#pragma unroll
+          for (int i = 0; i < 16; ++i) pk[i] = scale_bf16_pair(pk[i], alpha);
+          tmem_st16(tS + qq * 16, pk);
+        }
+      }
+      alpha_total *= alpha;
+      moved = true;
+      if (grow) m_ref = mxs;
+    }
+    // ---- P
+    const float nm = (PARTIAL && m_ref == -INFINITY) ? 0.f : -m_ref;
+    const uint64_t nm2 = pack2(nm, nm);
     uint32_t pk[16];
 #pragma unroll
     for (int i = 0; i < 16; ++i) {
@@ -112,12 +107,32 @@ __device__ __forceinline__ bool softmax_tile_step(uint32_t tS, uint32_t tO, int 
     }
     tmem_st16(tS + q4 * 16, pk);
   }
+  float l_tile;
   {
     float a0, a1, b0, b1;
     unpack2(add2(lacc[0], lacc[1]), a0, a1);
     unpack2(add2(lacc[2], lacc[3]), b0, b1);
-    l += (a0 + a1) + (b0 + b1);
+    l_tile = (a0 + a1) + (b0 + b1);
   }
+  bool o_waited = false;
+  if (moved) {
+    l *= alpha_total;
+    if (j > 0) {  // O(j-1) must be complete before it is rescaled
+      if (!wait_o()) return false;
+      o_waited = true;
+      tc_fence_after();
+#pragma unroll
+      for (int q4 = 0; q4 < 4; ++q4) {
+        uint32_t o[32];
+        tmem_ld32(tO + q4 * 32, o);
+        tc_wait_ld();
+#pragma unroll
+        for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha_total);
+        tmem_st32(tO + q4 * 32, o);
+      }
+    }
+  }
+  l += l_tile;
   tc_wait_st();
   // every phase of the O-complete barrier is waited on exactly once, in order, so a parity never aliases;
   // PV(j) queues behind PV(j-1) in the tensor pipe anyway, so this costs no overlap
