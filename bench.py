@@ -1,7 +1,7 @@
 #!/usr/bin/env python
 """Benchmark of the KV-cache attention hot path on B200.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg2] [--impl ours|reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg3_c512] [--impl ours|reference]
 
 One step = one pass of the whole hot path over one batch of seeded synthetic input:
 for a prefill workload every chunk is written to the cache and attends to it
@@ -42,7 +42,8 @@ def parse_args():
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="cfg2", choices=sorted(PREFILL) + sorted(BRANCH))
+    ap.add_argument("--workload", default="cfg3_c512", choices=sorted(PREFILL) + sorted(BRANCH),
+                    help="default: the largest single-GPU workload (4 x 8192-token GQA prompts, chunks of 512)")
     ap.add_argument("--no-extra", action="store_true", help="skip the short runs of the other workloads")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-graph", action="store_true", help="time eager launches instead of a CUDA-graph replay")
@@ -158,12 +159,11 @@ def timed_steps(step_fn, steps, warmup, flush, dist_barrier):
 class PrefillRun:
     """Device state and step function of a chunked-prefill workload."""
 
-    def __init__(self, ctx, w, device):
+    def __init__(self, ctx, w, device, data=None):
         import torch
         import paper_2504_08242_b200 as J
         self.ctx, self.w = ctx, w
-        q, k, v = w.make()
-        self.host = (q, k, v)
+        q, k, v = data if data is not None else w.make()
         qd, kd, vd = _dev(q, device), _dev(k, device), _dev(v, device)
         self.kc = torch.zeros(w.batch, w.kv_heads, w.capacity, w.head_dim, dtype=torch.bfloat16, device=device)
         self.vc = torch.zeros_like(self.kc)
@@ -413,23 +413,33 @@ def e2e_measure(run, steps, warmup, flush):
 
 # ----------------------------------------------------------------------------- CPU oracle legs
 
-def oracle_prefill_sample(w, kv_heads_used, threads):
-    """Runs the oracle (append + chunk attention for every chunk) on sequence 0 and the first
-    `kv_heads_used` KV heads with their query heads; returns (seconds, flops done)."""
+_SEQ0 = {}
+
+
+def oracle_prefill_sample(w, kv_heads_used, threads, n_chunks=None):
+    """Runs the oracle (append + chunk attention) on sequence 0, the first `kv_heads_used` KV heads with their query
+    heads and the first `n_chunks` chunks of the prompt (all by default); returns (seconds, flops done)."""
+    import dataclasses
     import oracle
     G = w.q_heads // w.kv_heads
-    q, k, v = w.make()
-    q = np.ascontiguousarray(q[:1, :, :kv_heads_used * G])
-    k = np.ascontiguousarray(k[:1, :, :kv_heads_used])
-    v = np.ascontiguousarray(v[:1, :, :kv_heads_used])
-    kc = np.zeros((1, kv_heads_used, w.capacity, w.head_dim), np.uint16)
+    chunks = w.chunks()[:n_chunks] if n_chunks else w.chunks()
+    tokens = chunks[-1][0] + chunks[-1][1]
+    # the generator is counter based: sequence 0 of the workload is the one-sequence workload's only sequence
+    w1 = dataclasses.replace(w, batch=1, chunk=1, name="")
+    if _SEQ0.get("key") != w1:
+        _SEQ0.update(key=w1, data=w1.make())  # kept: the same sample is timed several times
+    q, k, v = _SEQ0["data"]
+    q = np.ascontiguousarray(q[:1, :tokens, :kv_heads_used * G])
+    k = np.ascontiguousarray(k[:1, :tokens, :kv_heads_used])
+    v = np.ascontiguousarray(v[:1, :tokens, :kv_heads_used])
+    kc = np.zeros((1, kv_heads_used, tokens, w.head_dim), np.uint16)
     vc = np.zeros_like(kc)
     t0 = time.perf_counter()
-    for pos, n in w.chunks():
+    for pos, n in chunks:
         oracle.kv_append(kc, vc, k[:, pos:pos + n], v[:, pos:pos + n], pos=pos)
         oracle.chunk_prefill(q[:, pos:pos + n], kc, vc, pos, w.scale, n_threads=threads)
     dt = time.perf_counter() - t0
-    return dt, 4.0 * w.head_dim * kv_heads_used * G * w.pairs()
+    return dt, 4.0 * w.head_dim * kv_heads_used * G * (tokens * (tokens + 1) // 2)
 
 
 def oracle_branch_sample(w, n_steps, threads):
@@ -464,8 +474,16 @@ def cpu_leg(w, target_seconds):
         step = max(1, threads // G)  # whole multiples of the thread count keep every thread busy
         heads = int(max(step, min(w.kv_heads, (target_seconds / max(per_head, 1e-9)) // step * step)))
         heads = min(heads, w.kv_heads)
-        dt, fl = oracle_prefill_sample(w, heads, threads)
-        return fl / dt, f"sequence 0, KV heads 0..{heads - 1} of {w.kv_heads} with their query heads, all chunks", threads
+        # a long prompt whose smallest head set is still too much work: only its first chunks (the work grows with the
+        # square of the tokens covered)
+        n_chunks = len(w.chunks())
+        est = per_head * (heads + step - 1) // step if step else per_head
+        if est > 1.5 * target_seconds:
+            frac = (target_seconds / est) ** 0.5
+            n_chunks = int(max(1, min(n_chunks, round(frac * n_chunks))))
+        dt, fl = oracle_prefill_sample(w, heads, threads, n_chunks)
+        return (fl / dt, f"sequence 0, KV heads 0..{heads - 1} of {w.kv_heads} with their query heads, "
+                f"chunks 0..{n_chunks - 1} of {len(w.chunks())}", threads)
     dt1, b1 = oracle_branch_sample(w, 1, threads)
     n = int(max(1, min(w.steps, target_seconds / max(dt1, 1e-9))))
     dt, nb = oracle_branch_sample(w, n, threads)
@@ -518,7 +536,8 @@ def reference_arm(args, rank):
     # re-run the same sample K (+W) times
     if isinstance(w, synth.PrefillWorkload):
         heads = int(sample.split("..")[1].split(" ")[0]) + 1
-        fn = lambda: oracle_prefill_sample(w, heads, threads)
+        n_chunks = int(sample.split("..")[2].split(" ")[0]) + 1
+        fn = lambda: oracle_prefill_sample(w, heads, threads, n_chunks)
     else:
         n = int(sample.split("..")[1].split(" ")[0]) + 1
         fn = lambda: oracle_branch_sample(w, n, threads)
@@ -556,18 +575,137 @@ def whole_job_value(units_per_rank: float, world: int, ms_per_step: float, scale
     return world * units_per_rank / (ms_per_step * 1e-3) / scale
 
 
-# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) per launch of the dominant kernel, from one
-# ncu capture of that kernel on that workload.  A figure is only valid for the kernel build it was taken
-# on: set it to None when that kernel changes.
-NCU_TRAFFIC_BYTES_PER_LAUNCH = {
-    "cfg2": 21.06e6,       # prefill_tc_kernel, mean over the 8 chunk launches (compulsory: Q chunk + K/V rows 0..pos+n)
-    "cfg4": 31.54e6,       # branch_stream_kernel<128, 8, 2>, decode step 6 (31.6 MB algorithmic)
-    "cfg5": 28.08e6,       # branch_attn_kernel, the verification step (29.3 MB algorithmic)
+# ----------------------------------------------------------------------------- ncu traffic figures
+
+# Which profile summary carries the DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum per launch) of a
+# workload's dominant kernel, and which source files that kernel is built from.  A summary is stamped with the
+# hash of those sources at the time of its capture; when the kernel has changed since, the figure is void and
+# the bench line says null.
+CSRC = os.path.join(ROOT, "paper_2504_08242_b200", "csrc")
+TC_SOURCES = ["tc_common.cuh", "tc_softmax.cuh", "common.cuh"]
+TRAFFIC_PROFILES = {
+    "cfg2": ("prefill_tc_kernel_cfg2.md", ["prefill_tc.cu"] + TC_SOURCES),
+    "cfg3_c128": ("prefill_tc_kernel_cfg3_c512.md", ["prefill_tc.cu"] + TC_SOURCES),
+    "cfg3_c512": ("prefill_tc_kernel_cfg3_c512.md", ["prefill_tc.cu"] + TC_SOURCES),
+    "cfg3_c1024": ("prefill_tc_kernel_cfg3_c512.md", ["prefill_tc.cu"] + TC_SOURCES),
+    "cfg4": ("branch_stream_kernel_cfg4.md", ["branch_stream.cu", "tc_common.cuh", "common.cuh"]),
+    "cfg5": ("branch_tc_kernel_cfg5.md", ["branch_tc.cu"] + TC_SOURCES),
 }
+
+
+def kernel_source_hash(files):
+    import hashlib
+    h = hashlib.sha1()
+    for f in files:
+        with open(os.path.join(CSRC, f), "rb") as fh:
+            h.update(fh.read())
+    return h.hexdigest()[:16]
+
+
+def ncu_traffic(name, launch_bytes=None):
+    """(bytes per launch or None, where it comes from).  The summary holds the lines
+    ``kernel_source_sha1: <hash>`` and ``dram_bytes_per_launch[<workload>]: <bytes>``; for the prefill sweeps the
+    capture is of one launch of the sweep and the line is ``dram_bytes_per_algorithmic_byte: <ratio>``, scaled
+    here by the workload's mean compulsory bytes per launch (traffic grows in proportion to the K/V rows read)."""
+    import re
+    prof, files = TRAFFIC_PROFILES.get(name, (None, None))
+    if prof is None:
+        return None, "no capture"
+    path = os.path.join(ROOT, "profiles", prof)
+    if not os.path.exists(path):
+        return None, f"profiles/{prof} missing"
+    text = open(path).read()
+    m = re.search(r"kernel_source_sha1:\s*([0-9a-f]+)", text)
+    if not m or m.group(1) != kernel_source_hash(files):
+        return None, f"profiles/{prof}: taken on an older build of the kernel"
+    m = re.search(r"dram_bytes_per_launch\[%s\]:\s*([0-9.eE+]+)" % re.escape(name), text)
+    if m:
+        return float(m.group(1)), f"profiles/{prof}"
+    m = re.search(r"dram_bytes_per_algorithmic_byte:\s*([0-9.eE+]+)", text)
+    if m and launch_bytes:
+        return float(m.group(1)) * launch_bytes, f"profiles/{prof} (ratio measured on one launch x this workload's mean compulsory bytes per launch)"
+    return None, f"profiles/{prof}: no figure for {name}"
+
+
+def prefill_launch_bytes(w):
+    """Compulsory DRAM bytes of an average chunk launch: Q read, the chunk's K/V read and written to the cache,
+    the cached rows [0, pos) read, fp32 output written."""
+    tot = 0
+    for pos, n in w.chunks():
+        kv_row = w.kv_heads * w.head_dim * 2
+        tot += w.batch * (n * w.q_heads * w.head_dim * (2 + 4) + 2 * kv_row * (2 * n + pos))
+    return tot / len(w.chunks())
+
+
+# ----------------------------------------------------------------------------- one workload on the GPU
+
+def run_workload(ctx, device, name, w, steps, warmup, flush, barrier, world, peaks, peak_kind, use_graph=True,
+                 prefill_data=None, with_e2e=True, rank=0):
+    """Times one workload and returns the fields of its bench entry: value, ms_per_step, clocks (sampled during its
+    own timed region), gpu_launches, roofline, e2e."""
+    import torch
+    is_prefill = isinstance(w, synth.PrefillWorkload)
+    run = PrefillRun(ctx, w, device, data=prefill_data) if is_prefill else branch_run(ctx, w, device)
+    sampler = ClockSampler(device.index or 0)
+    sampler.start()
+    m = measure(run, steps, warmup, flush, barrier, use_graph=use_graph, sampler=sampler)
+    clocks = sampler.stop(*m["sample_range"])
+    assert ctx.poll_device_status() == 0
+    ms_per_step = max_over_ranks(m["ms_per_step"], world, device)
+    value = whole_job_value(run.units(), world, ms_per_step, scale_of(w))
+    if is_prefill:
+        achieved = run.units() / (m["attn_ms_per_step"] * 1e-3) / 1e12
+        peak = peaks["bf16_tflops"]
+        traffic, traffic_from = ncu_traffic(name, prefill_launch_bytes(w))
+        roofline = {"bound": "tensor", "kernel": "chunk_prefill_attn", "achieved": achieved, "peak": peak,
+                    "unit": "TFLOP/s", "frac": achieved / peak, "peak_kind": f"{peak_kind} burst bf16",
+                    "frac_of_sustained": achieved / peaks["bf16_tflops_sustained"],
+                    "avg_launch_ms": m["attn_ms_per_launch"], "avg_launch_from": m["attn_time_source"],
+                    "traffic": traffic, "traffic_from": traffic_from,
+                    "traffic_unit": "bytes per launch (ncu dram read+write)"}
+    else:
+        achieved = run.units() / (m["attn_ms_per_step"] * 1e-3) / 1e9
+        peak = peaks["hbm_gbs"]
+        traffic, traffic_from = ncu_traffic(name)
+        roofline = {"bound": "hbm", "kernel": "branch_attn", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                    "frac": achieved / peak, "peak_kind": f"{peak_kind} copy", "avg_launch_ms": m["attn_ms_per_launch"],
+                    "avg_launch_from": m["attn_time_source"], "traffic": traffic, "traffic_from": traffic_from,
+                    "traffic_unit": "bytes per launch (ncu dram read+write)"}
+        if rank == 0:
+            n_launch = run.attn_launches_per_step()
+            roofline["plain_read"] = plain_read_floor(ctx, device, run.units() / n_launch, max(n_launch, 16), flush)
+    extra = {} if is_prefill else {"cache_copies_rotated": run.copies, "passes_per_step": run.passes,
+                                   "calls_per_step": run.attn_launches_per_step()}
+    if not use_graph:
+        extra["launch"] = "eager"
+    entry = {"value": value, "unit": unit_of(w), "steps": steps, "warmup": warmup, "ms_per_step": ms_per_step,
+             "config": config_of(name, w, extra), "clocks": clocks, "gpu_launches": m["launches_per_step"] * steps,
+             "roofline": roofline}
+    if with_e2e:
+        e2e_ms, h2d, d2h = e2e_measure(run, max(3, steps // 4), 2, flush)
+        entry["e2e"] = {"value": whole_job_value(run.units(), world, max_over_ranks(e2e_ms, world, device), scale_of(w)),
+                        "unit": unit_of(w), "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}
+    del run
+    torch.cuda.empty_cache()
+    return entry
+
+
+def relaunch_under_torchrun(args):
+    """`--gpus N` without a launcher: start one rank per GPU under torchrun (standalone, local rendezvous) and pass
+    its output and exit status through."""
+    import socket
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        port = sk.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={args.gpus}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    return subprocess.call(cmd)
 
 
 def main():
     args = parse_args()
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        return relaunch_under_torchrun(args)
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
@@ -595,56 +733,38 @@ def main():
     flush = Flusher(device)
     name = args.workload
     w = make_workload(name)
-    is_prefill = isinstance(w, synth.PrefillWorkload)
-    # branch workloads fit in L2: rotate the decode steps over independent cache copies so each reads cold data
-    run = PrefillRun(ctx, w, device) if is_prefill else branch_run(ctx, w, device)
+    # the three chunk sizes of the long-prompt workload share one prompt: generate it once
+    shared = {}
 
-    sampler = ClockSampler(local_rank)
-    sampler.start()
-    m = measure(run, args.steps, args.warmup, flush, barrier, use_graph=not args.no_graph, sampler=sampler)
-    clocks = sampler.stop(*m["sample_range"])
-    assert ctx.poll_device_status() == 0
+    def data_for(n, wl):
+        if not isinstance(wl, synth.PrefillWorkload):
+            return None
+        key = (wl.seed, wl.batch, wl.q_heads, wl.kv_heads, wl.head_dim, wl.seq_len)
+        if key not in shared:
+            shared.clear()  # one prompt resident at a time
+            shared[key] = wl.make()
+        return shared[key]
 
-    ms_per_step = max_over_ranks(m["ms_per_step"], world, device)
-    value = whole_job_value(run.units(), world, ms_per_step, scale_of(w))
-
-    e2e_ms, h2d, d2h = e2e_measure(run, max(3, args.steps // 4), 2, flush)
-    e2e_value = whole_job_value(run.units(), world, max_over_ranks(e2e_ms, world, device), scale_of(w))
-
-    if is_prefill:
-        achieved = run.units() / (m["attn_ms_per_step"] * 1e-3) / 1e12
-        peak = peaks["bf16_tflops"]
-        roofline = {"bound": "tensor", "kernel": "chunk_prefill_attn", "achieved": achieved, "peak": peak,
-                    "unit": "TFLOP/s", "frac": achieved / peak, "peak_kind": f"{peak_kind} burst bf16",
-                    "frac_of_sustained": achieved / peaks["bf16_tflops_sustained"],
-                    "avg_launch_ms": m["attn_ms_per_launch"], "avg_launch_from": m["attn_time_source"],
-                    "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH.get(name),
-                    "traffic_unit": "bytes per launch (ncu dram read+write)"}
-    else:
-        achieved = run.units() / (m["attn_ms_per_step"] * 1e-3) / 1e9
-        peak = peaks["hbm_gbs"]
-        roofline = {"bound": "hbm", "kernel": "branch_attn", "achieved": achieved, "peak": peak, "unit": "GB/s",
-                    "frac": achieved / peak, "peak_kind": f"{peak_kind} copy", "avg_launch_ms": m["attn_ms_per_launch"],
-                    "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH.get(name),
-                    "traffic_unit": "bytes per launch (ncu dram read+write)"}
-        if rank == 0:
-            n_launch = run.attn_launches_per_step()
-            roofline["plain_read"] = plain_read_floor(ctx, device, run.units() / n_launch, max(n_launch, 16), flush)
-
-    line = {"metric": METRIC, "value": value, "unit": unit_of(w), "n_gpus": world, "steps": args.steps,
-            "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
-            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-            "config": config_of(name, w, dict({} if is_prefill else {"cache_copies_rotated": run.copies, "passes_per_step": run.passes,
-                                                                    "calls_per_step": run.attn_launches_per_step()},
-                                              **({"launch": "eager"} if args.no_graph else {}))),
-            "clocks": clocks, "gpu_launches": m["launches_per_step"] * args.steps,
-            "e2e": {"value": e2e_value, "unit": unit_of(w), "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
-            "roofline": roofline}
+    head = run_workload(ctx, device, name, w, args.steps, args.warmup, flush, barrier, world, peaks, peak_kind,
+                        use_graph=not args.no_graph, prefill_data=data_for(name, w), rank=rank)
+    line = {"metric": METRIC, "value": head["value"], "unit": head["unit"], "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": head["ms_per_step"], "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic", "config": head["config"], "clocks": head["clocks"],
+            "gpu_launches": head["gpu_launches"], "e2e": head["e2e"], "roofline": head["roofline"]}
 
     if rank == 0 and world == 1 and not args.no_extra:
-        line["other_workloads"] = other_workloads(ctx, device, flush, peaks, skip=name, run=run)
+        # the other workloads, each a full entry of its own (same steps and warm-up, its own clock record)
+        others = {}
+        for other in ("cfg3_c1024", "cfg3_c128", "cfg3_c512", "cfg2", "cfg4", "cfg5"):
+            if other == name:
+                continue
+            ow = make_workload(other)
+            others[other] = run_workload(ctx, device, other, ow, max(args.steps, 20), max(args.warmup, 3), flush,
+                                         lambda: None, 1, peaks, peak_kind, prefill_data=data_for(other, ow),
+                                         with_e2e=False)
+        line["other_workloads"] = others
+    shared.clear()
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        del run
         rate, sample, threads = cpu_leg(w, args.cpu_seconds)
         line["cpu_baseline"] = {"value": rate / scale_of(w), "unit": unit_of(w), "cores": threads, "kind": "oracle",
                                 "sample": sample}
@@ -654,43 +774,6 @@ def main():
         dist.barrier()
         dist.destroy_process_group()
     return 0
-
-
-def other_workloads(ctx, device, flush, peaks, skip, run=None):
-    """Short runs of the remaining workloads, reported beside the headline (each: a few steps)."""
-    import torch
-    out = {}
-    plan = [("cfg2", 10), ("cfg3_c512", 2), ("cfg3_c1024", 2), ("cfg3_c128", 2), ("cfg4", 5), ("cfg5", 20)]
-    for name, steps in plan:
-        if name == skip:
-            continue
-        w = make_workload(name)
-        torch.cuda.empty_cache()
-        if isinstance(w, synth.PrefillWorkload):
-            r = PrefillRun(ctx, w, device)
-            m = measure(r, steps, 3, flush, lambda: None)
-            tf = r.units() / (m["ms_per_step"] * 1e-3) / 1e12
-            ka = r.units() / (m["attn_ms_per_step"] * 1e-3) / 1e12
-            out[name] = {"value": tf, "unit": "TFLOP/s", "ms_per_step": m["ms_per_step"], "attn_kernel_tflops": ka,
-                         "attn_frac_of_bf16_peak": ka / peaks["bf16_tflops"],
-                         "attn_frac_of_bf16_sustained": ka / peaks["bf16_tflops_sustained"], "steps": steps}
-        else:
-            res = {}
-            for label in ("cold", "warm"):
-                r = branch_run(ctx, w, device, cold=label == "cold")
-                m = measure(r, steps, 3, flush, lambda: None)
-                gb = r.units() / (m["attn_ms_per_step"] * 1e-3) / 1e9
-                res[label] = {"attn_gbs": gb, "frac_of_hbm_peak": gb / peaks["hbm_gbs"],
-                              "step_gbs": r.units() / (m["ms_per_step"] * 1e-3) / 1e9,
-                              "attn_us_per_launch": 1e3 * m["attn_ms_per_launch"], "ms_per_step": m["ms_per_step"]}
-                if label == "cold":
-                    n_launch = r.attn_launches_per_step()
-                    res["plain_read"] = plain_read_floor(ctx, device, r.units() / n_launch, max(n_launch, 16), flush)
-                del r
-            res["unit"] = "GB/s"
-            res["steps"] = steps
-            out[name] = res
-    return out
 
 
 if __name__ == "__main__":

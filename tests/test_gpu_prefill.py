@@ -139,14 +139,8 @@ def test_results_are_run_to_run_identical(ctx):
     assert np.array_equal(a, b)
 
 
-@pytest.mark.parametrize("chunk", [128, 512, 1024])
-def test_cfg3_gqa_long_prompt_sampled_rows(ctx, chunk):
-    """Full 4 x 8192-token GQA prompt on the GPU in the launch configuration the benchmark
-    times; the oracle evaluates sampled (sequence, head, row) outputs one by one."""
-    w = synth.cfg3(chunk)
-    q, k, v = w.make()
-    out = run_gpu_prefill(ctx, q, k, v, [n for _, n in w.chunks()], w.capacity, w.scale, poison=False)[0]
-    assert np.isfinite(out).all()
+def _cfg3_sampled_rows(w, q, k, v, out, chunk):
+    """The oracle evaluates sampled (sequence, head, row) outputs of the full-size workload one by one."""
     G = w.q_heads // w.kv_heads
     rows = [(0, 0, 0), (3, 31, 8191), (1, 5, chunk - 1), (2, 17, chunk), (0, 9, 4095), (3, 2, 8191 - chunk)]
     pick = synth.uniform_ints(99, 1, 3 * 58, 0, 1 << 30).reshape(-1, 3)
@@ -159,6 +153,32 @@ def test_cfg3_gqa_long_prompt_sampled_rows(ctx, chunk):
         ref.append(o)
         got.append(out[b, i, h])
     assert_close(np.array(got), np.array(ref), w.name)
+
+
+@pytest.mark.parametrize("chunk", [128, 512, 1024])
+def test_cfg3_gqa_long_prompt_sampled_rows(ctx, chunk):
+    """Full 4 x 8192-token GQA prompt on the GPU through the two-call form (jupiter_kv_append, then
+    jupiter_chunk_prefill_attn per chunk)."""
+    w = synth.cfg3(chunk)
+    q, k, v = w.make()
+    out = run_gpu_prefill(ctx, q, k, v, [n for _, n in w.chunks()], w.capacity, w.scale, poison=False)[0]
+    assert np.isfinite(out).all()
+    _cfg3_sampled_rows(w, q, k, v, out, chunk)
+
+
+@pytest.mark.parametrize("chunk", [128, 512, 1024])
+def test_cfg3_fused_sampled_rows(ctx, chunk):
+    """The same workload in the launch configuration the benchmark times: one jupiter_chunk_prefill_append_attn call
+    per chunk (batch 4, GQA, 64 / 16 / 8 launches walking up to 64 KV tiles).  Sampled outputs against the oracle,
+    and the final caches bit for bit against the prompt's K/V (dead rows, poisoned beforehand, included)."""
+    from tests.helpers import token_to_cache
+    w = synth.cfg3(chunk)
+    q, k, v = w.make()
+    cap = w.capacity + 128  # rows above the prompt stay poisoned
+    out, kc, vc = run_gpu_prefill(ctx, q, k, v, [n for _, n in w.chunks()], cap, w.scale, poison=True, fused=True)
+    assert np.isfinite(out).all()
+    _cfg3_sampled_rows(w, q, k, v, out, chunk)
+    assert np.array_equal(kc, token_to_cache(k, cap, 0x7FC0)) and np.array_equal(vc, token_to_cache(v, cap, 0x7F80))
 
 
 def test_prefill_argument_errors(ctx):
