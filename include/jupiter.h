@@ -204,6 +204,33 @@ jupiter_status jupiter_branch_append_attn(jupiter_ctx* ctx, const void* q, const
                                           int32_t max_suffix_len, int32_t n_branches, int32_t q_heads,
                                           int32_t q_len, float scale, float* out, float* lse, void* stream);
 
+/* One decoding / verification step for several decoder layers in one call (Sec. V-A, Fig. 7 steps 3-5 run in
+ * every decoder layer of a stage; Sec. V-B: every layer keeps its own shared prompt KVCache and per-request
+ * KVCaches).  Layer l has its own query block, K/V block, prefix cache, suffix cache and outputs; all layers have
+ * the same geometry (head counts, head_dim, capacities, strides), the same branch lengths and the same scale.
+ * Same result, layer by layer, as n_layers calls of jupiter_branch_append_attn -- the layers must not depend on one
+ * another's outputs inside the call (their Q/K/V blocks are ready beforehand) -- but the layers share launches: with
+ * few stacked query rows per kv head (decode) up to 16 layers run as ONE kernel launch, so the time between
+ * dependent launches is paid once per 16 layers instead of once per layer; shapes that take the other kernels are
+ * enqueued layer by layer.
+ *   layers: HOST array of n_layers entries (read during the call only); prefix may be NULL when prefix_len == 0;
+ *           lse may be NULL.  Other arguments and errors as for jupiter_branch_append_attn; every layer's
+ *           descriptors are checked before anything is enqueued, and a layer whose geometry differs from
+ *           layer 0's is JUPITER_ERR_INVALID_ARG. */
+typedef struct {
+  const void* q;                  /* [n_branches][q_len][q_heads][D] bf16 */
+  const void* k_new;              /* [n_branches][q_len][kv_heads][D] bf16 */
+  const void* v_new;
+  const jupiter_kv_cache* prefix; /* batch == 1 */
+  const jupiter_kv_cache* suffix; /* batch == n_branches */
+  float* out;                     /* [n_branches][q_len][q_heads][D] fp32 */
+  float* lse;                     /* nullable: [n_branches][q_heads][q_len] */
+} jupiter_branch_layer;
+jupiter_status jupiter_branch_append_attn_layers(jupiter_ctx* ctx, const jupiter_branch_layer* layers,
+                                                 int32_t n_layers, int32_t prefix_len, const int32_t* d_suffix_len,
+                                                 int32_t max_suffix_len, int32_t n_branches, int32_t q_heads,
+                                                 int32_t q_len, float scale, void* stream);
+
 /* Tuning and testing aid; the paper has no counterpart.  The branch calls (jupiter_branch_attn, _tree,
  * jupiter_branch_append_attn) pick one of three kernels from the shape: a streaming kernel for few stacked
  * query rows per kv head (decode), a tensor-core kernel (tcgen05 / TMEM) for many rows with head_dim 128, and a

@@ -33,6 +33,7 @@ EXPORTS = (
     "jupiter_plan_sequence_partition", "jupiter_branch_attn_tree", "jupiter_branch_prefill_attn",
     "jupiter_chunk_prefill_append_attn", "jupiter_branch_append_attn", "jupiter_read_probe",
     "jupiter_kv_compact", "jupiter_wait_probe", "jupiter_select_branch_kernel",
+    "jupiter_branch_append_attn_layers",
 )
 
 
@@ -40,6 +41,11 @@ class jupiter_kv_cache(ctypes.Structure):
     _fields_ = [("k", c_void_p), ("v", c_void_p), ("batch", c_int32), ("kv_heads", c_int32),
                 ("capacity", c_int32), ("head_dim", c_int32), ("stride_batch", c_int64),
                 ("stride_head", c_int64), ("stride_row", c_int64)]
+
+
+class jupiter_branch_layer(ctypes.Structure):
+    _fields_ = [("q", c_void_p), ("k_new", c_void_p), ("v_new", c_void_p), ("prefix", ctypes.POINTER(jupiter_kv_cache)),
+                ("suffix", ctypes.POINTER(jupiter_kv_cache)), ("out", c_void_p), ("lse", c_void_p)]
 
 
 class JupiterError(RuntimeError):
@@ -72,6 +78,9 @@ def _load() -> ctypes.CDLL:
     lib.jupiter_launch_count.restype = ctypes.c_uint64
     lib.jupiter_kv_compact.argtypes = [c_void_p, P(jupiter_kv_cache), c_int32, c_void_p, c_void_p, c_void_p, c_void_p]
     lib.jupiter_kv_compact.restype = ctypes.c_int
+    lib.jupiter_branch_append_attn_layers.argtypes = [c_void_p, P(jupiter_branch_layer), c_int32, c_int32, c_void_p,
+                                                      c_int32, c_int32, c_int32, c_int32, c_float, c_void_p]
+    lib.jupiter_branch_append_attn_layers.restype = ctypes.c_int
     lib.jupiter_select_branch_kernel.argtypes = [c_void_p, ctypes.c_int]
     lib.jupiter_select_branch_kernel.restype = ctypes.c_int
     lib.jupiter_wait_probe.argtypes = [c_void_p, c_int64, c_void_p]
@@ -209,6 +218,20 @@ class Context:
                                                    ctypes.byref(suffix), _ptr(d_suffix_len), max_suffix_len,
                                                    n_branches, q_heads, q_len, scale, _ptr(out), _ptr(lse),
                                                    _stream(stream)))
+
+    def branch_append_attn_layers(self, layers, prefix_len: int, d_suffix_len, max_suffix_len: int, n_branches: int,
+                                  q_heads: int, q_len: int, scale: float, stream=None):
+        """layers: sequence of (q, k_new, v_new, prefix descriptor or None, suffix descriptor, out, lse or None)."""
+        arr = (jupiter_branch_layer * len(layers))()
+        for i, (q, kn, vn, pfx, sfx, out, lse) in enumerate(layers):
+            arr[i].q, arr[i].k_new, arr[i].v_new = q.data_ptr(), kn.data_ptr(), vn.data_ptr()
+            arr[i].prefix = ctypes.pointer(pfx) if pfx is not None else None
+            arr[i].suffix = ctypes.pointer(sfx)
+            arr[i].out = out.data_ptr()
+            arr[i].lse = lse.data_ptr() if lse is not None else None
+        self._check(lib.jupiter_branch_append_attn_layers(self._h, arr, len(layers), prefix_len, _ptr(d_suffix_len),
+                                                          max_suffix_len, n_branches, q_heads, q_len, scale,
+                                                          _stream(stream)))
 
     def branch_prefill_attn(self, q, prefix: jupiter_kv_cache, prefix_len: int, cache: jupiter_kv_cache,
                             q_heads: int, q_len: int, pos: int, scale: float, out, lse=None, stream=None):

@@ -3,6 +3,7 @@
 #include <cstdio>
 #include <cstring>
 #include <new>
+#include <vector>
 
 #include "../../include/jupiter.h"
 #include "host_checks.h"
@@ -340,6 +341,67 @@ static jupiter_status branch_attn_impl(jupiter_ctx* ctx, const void* q, const ju
                            static_cast<const bf16*>(v_new));
   ctx->launches += li.launches;
   return e == cudaSuccess ? JUPITER_OK : cuda_fail(ctx, e, "branch_attn");
+}
+
+jupiter_status jupiter_branch_append_attn_layers(jupiter_ctx* ctx, const jupiter_branch_layer* layers,
+                                                 int32_t n_layers, int32_t prefix_len, const int32_t* d_suffix_len,
+                                                 int32_t max_suffix_len, int32_t n_branches, int32_t q_heads,
+                                                 int32_t q_len, float scale, void* stream) {
+  if (!ctx || !layers || n_layers <= 0 || !d_suffix_len) return JUPITER_ERR_INVALID_ARG;
+  if (prefix_len < 0 || n_branches <= 0 || q_heads <= 0 || q_len <= 0) return JUPITER_ERR_INVALID_ARG;
+  if (q_len > 16) return JUPITER_ERR_UNSUPPORTED;
+  if (!jup::scale_ok(scale)) return JUPITER_ERR_INVALID_ARG;
+  // every layer is checked before anything is enqueued
+  CacheView sfx0, pfx0;
+  std::vector<jup::BranchLayerTensors> t(static_cast<size_t>(n_layers));
+  for (int l = 0; l < n_layers; ++l) {
+    const jupiter_branch_layer& L = layers[l];
+    if (!L.q || !L.k_new || !L.v_new || !L.out) return JUPITER_ERR_INVALID_ARG;
+    if (!aligned16(L.q) || !aligned16(L.k_new) || !aligned16(L.v_new) || !aligned16(L.out)) return JUPITER_ERR_ALIGNMENT;
+    CacheView sfx;
+    jupiter_status s = check_cache(L.suffix, &sfx);
+    if (s != JUPITER_OK) return s;
+    CacheView pfx = sfx;
+    if (prefix_len > 0) {
+      s = check_cache(L.prefix, &pfx);
+      if (s != JUPITER_OK) return s;
+      if (pfx.batch != 1 || pfx.kv_heads != sfx.kv_heads || pfx.head_dim != sfx.head_dim) return JUPITER_ERR_INVALID_ARG;
+      if (prefix_len > pfx.capacity) return JUPITER_ERR_OUT_OF_RANGE;
+    }
+    if (n_branches != sfx.batch || q_heads % sfx.kv_heads != 0) return JUPITER_ERR_INVALID_ARG;
+    if (max_suffix_len < q_len || max_suffix_len > sfx.capacity) return JUPITER_ERR_OUT_OF_RANGE;
+    if (l == 0) {
+      sfx0 = sfx;
+      pfx0 = pfx;
+    } else {
+      auto same = [](const CacheView& a, const CacheView& b) {
+        return a.batch == b.batch && a.kv_heads == b.kv_heads && a.capacity == b.capacity && a.head_dim == b.head_dim &&
+               a.sb == b.sb && a.sh == b.sh && a.sr == b.sr;
+      };
+      if (!same(sfx, sfx0) || (prefix_len > 0 && !same(pfx, pfx0))) return JUPITER_ERR_INVALID_ARG;
+    }
+    t[l] = jup::BranchLayerTensors{static_cast<const bf16*>(L.q), static_cast<const bf16*>(L.k_new),
+                                   static_cast<const bf16*>(L.v_new), pfx.k, pfx.v, sfx.k, sfx.v, L.out, L.lse};
+  }
+  if (ctx->branch_kernel == JUPITER_BRANCH_AUTO &&
+      jup::branch_stream_preferred(n_branches, q_heads, sfx0.kv_heads, q_len, ctx->sm_count)) {
+    DeviceGuard guard(ctx->device);
+    jup::LaunchInfo li{ctx->sm_count, 0};
+    cudaError_t e = jup::launch_branch_stream_layers(t.data(), n_layers, pfx0, prefix_len, sfx0, d_suffix_len,
+                                                     max_suffix_len, n_branches, q_heads, q_len, scale,
+                                                     static_cast<cudaStream_t>(stream), li);
+    ctx->launches += li.launches;
+    return e == cudaSuccess ? JUPITER_OK : cuda_fail(ctx, e, "branch_append_attn_layers");
+  }
+  // the other kernels take the layers one by one (arguments are known to be valid; a layer can still find the
+  // context's scratch too small, before its own launch)
+  for (int l = 0; l < n_layers; ++l) {
+    const jupiter_branch_layer& L = layers[l];
+    jupiter_status s = branch_attn_impl(ctx, L.q, L.prefix, prefix_len, L.suffix, d_suffix_len, nullptr, max_suffix_len,
+                                        n_branches, q_heads, q_len, scale, L.out, L.lse, stream, L.k_new, L.v_new);
+    if (s != JUPITER_OK) return s;
+  }
+  return JUPITER_OK;
 }
 
 jupiter_status jupiter_branch_append_attn(jupiter_ctx* ctx, const void* q, const void* k_new, const void* v_new,

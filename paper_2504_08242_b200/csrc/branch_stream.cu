@@ -24,6 +24,8 @@
 // Fused KVCache write: with k_new / v_new the rows of this step's block are read from there
 // (they are not in the cache yet) and the warp that fetched them stores them into the suffix
 // rows [L_b - q_len, L_b) from shared memory.
+#include <algorithm>
+
 #include "host_checks.h"
 #include "kernels.h"
 #include "tc_common.cuh"
@@ -44,6 +46,24 @@ struct StreamParams {
   float scale_log2;
   float* out;
   float* lse;
+};
+
+// Several independent problems of the same geometry and lengths (the decoder layers of a step) in one launch:
+// blockIdx.y picks the problem, whose tensors replace the ones in StreamParams.
+struct StreamLayerPtrs {
+  const bf16* q;
+  const bf16* k_new;
+  const bf16* v_new;
+  const bf16* pk;
+  const bf16* pv;
+  const bf16* sk;
+  const bf16* sv;
+  float* out;
+  float* lse;
+};
+struct StreamLayers {
+  int n;  // 0: a plain launch, the tensors of StreamParams are used
+  StreamLayerPtrs l[kBranchMaxLayersPerLaunch];
 };
 
 template <int D, int NW, int ST>
@@ -77,7 +97,21 @@ __device__ __forceinline__ void st_cluster_f2(uint32_t addr, float2 v) {
 __device__ __forceinline__ int clampi(int v, int lo, int hi) { return v < lo ? lo : (v > hi ? hi : v); }
 
 template <int D, int NW, int ST>
-__global__ void __launch_bounds__(NW * 32, kStreamCtasPerSm) branch_stream_kernel(StreamParams p) {
+__global__ void __launch_bounds__(NW * 32, kStreamCtasPerSm)
+branch_stream_kernel(const StreamParams p_in, const __grid_constant__ StreamLayers layers) {
+  StreamParams p = p_in;
+  if (layers.n > 0) {
+    const StreamLayerPtrs& l = layers.l[blockIdx.y];
+    p.q = l.q;
+    p.k_new = l.k_new;
+    p.v_new = l.v_new;
+    p.prefix.k = l.pk;
+    p.prefix.v = l.pv;
+    p.suffix.k = l.sk;
+    p.suffix.v = l.sv;
+    p.out = l.out;
+    p.lse = l.lse;
+  }
   using Cfg = StreamCfg<D, NW, ST>;
   constexpr int CH = Cfg::CH;
   constexpr unsigned FULL = 0xffffffffu;
@@ -472,7 +506,8 @@ __global__ void __launch_bounds__(NW * 32, kStreamCtasPerSm) branch_stream_kerne
 }
 
 template <int D, int NW, int ST>
-static cudaError_t launch_stream_d(const StreamParams& p, int units, cudaStream_t st, LaunchInfo& li) {
+static cudaError_t launch_stream_d(const StreamParams& p, const StreamLayers& layers, int units, cudaStream_t st,
+                                   LaunchInfo& li) {
   using Cfg = StreamCfg<D, NW, ST>;
   static PerDeviceOnce attr_done;
   if (!attr_done.done()) {
@@ -485,8 +520,9 @@ static cudaError_t launch_stream_d(const StreamParams& p, int units, cudaStream_
     attr_done.set();
   }
   li.launches += 1;
-  return launch_pdl_cluster(branch_stream_kernel<D, NW, ST>, dim3(static_cast<unsigned>(units * p.cluster)),
-                            dim3(Cfg::THREADS), Cfg::SMEM_BYTES, st, static_cast<unsigned>(p.cluster), p);
+  return launch_pdl_cluster(branch_stream_kernel<D, NW, ST>,
+                            dim3(static_cast<unsigned>(units * p.cluster), static_cast<unsigned>(layers.n > 0 ? layers.n : 1)),
+                            dim3(Cfg::THREADS), Cfg::SMEM_BYTES, st, static_cast<unsigned>(p.cluster), p, layers);
 }
 
 bool branch_stream_preferred(int n_branches, int q_heads, int kv_heads, int q_len, int sm_count) {
@@ -497,10 +533,11 @@ bool branch_stream_preferred(int n_branches, int q_heads, int kv_heads, int q_le
   return tiles == 1 || tiles * kv_heads <= sm_count;
 }
 
-cudaError_t launch_branch_stream(const bf16* q, const CacheView& prefix, int prefix_len, const CacheView& suffix,
+static cudaError_t launch_stream(const bf16* q, const CacheView& prefix, int prefix_len, const CacheView& suffix,
                                  const int32_t* d_suffix_len, const uint32_t* d_tree_mask, int max_suffix_len,
                                  int n_branches, int q_heads, int q_len, float scale, float* out, float* lse,
-                                 cudaStream_t st, LaunchInfo& li, const bf16* k_new, const bf16* v_new) {
+                                 cudaStream_t st, LaunchInfo& li, const bf16* k_new, const bf16* v_new,
+                                 const StreamLayers& layers) {
   StreamParams p;
   p.q = q;
   p.prefix = prefix;
@@ -521,7 +558,7 @@ cudaError_t launch_branch_stream(const bf16* q, const CacheView& prefix, int pre
   p.out = out;
   p.lse = lse;
   const int units = suffix.kv_heads * p.row_tiles;
-  // the largest portable cluster that keeps every CTA resident at once
+  // the largest portable cluster that keeps every CTA (of one problem) resident at once
   int c = 1;
   while (c < 8 && units * c * 2 <= li.sm_count * kStreamCtasPerSm) c *= 2;
   // no more CTAs than 16-key chunks of work per unit warrant
@@ -529,8 +566,37 @@ cudaError_t launch_branch_stream(const bf16* q, const CacheView& prefix, int pre
   while (c > 1 && chunks < static_cast<int64_t>(c) * 8) c /= 2;
   p.cluster = c;
   p.cluster_log2 = c == 8 ? 3 : (c == 4 ? 2 : (c == 2 ? 1 : 0));
-  if (suffix.head_dim == 128) return launch_stream_d<128, kStreamWarps, kStreamStages>(p, units, st, li);
-  return launch_stream_d<64, kStreamWarps, kStreamStages>(p, units, st, li);
+  if (suffix.head_dim == 128) return launch_stream_d<128, kStreamWarps, kStreamStages>(p, layers, units, st, li);
+  return launch_stream_d<64, kStreamWarps, kStreamStages>(p, layers, units, st, li);
+}
+
+cudaError_t launch_branch_stream(const bf16* q, const CacheView& prefix, int prefix_len, const CacheView& suffix,
+                                 const int32_t* d_suffix_len, const uint32_t* d_tree_mask, int max_suffix_len,
+                                 int n_branches, int q_heads, int q_len, float scale, float* out, float* lse,
+                                 cudaStream_t st, LaunchInfo& li, const bf16* k_new, const bf16* v_new) {
+  StreamLayers none;
+  none.n = 0;
+  return launch_stream(q, prefix, prefix_len, suffix, d_suffix_len, d_tree_mask, max_suffix_len, n_branches, q_heads,
+                       q_len, scale, out, lse, st, li, k_new, v_new, none);
+}
+
+cudaError_t launch_branch_stream_layers(const BranchLayerTensors* layers, int n_layers, const CacheView& prefix,
+                                        int prefix_len, const CacheView& suffix, const int32_t* d_suffix_len,
+                                        int max_suffix_len, int n_branches, int q_heads, int q_len, float scale,
+                                        cudaStream_t st, LaunchInfo& li) {
+  for (int first = 0; first < n_layers; first += kBranchMaxLayersPerLaunch) {
+    StreamLayers batch;
+    batch.n = std::min(kBranchMaxLayersPerLaunch, n_layers - first);
+    for (int i = 0; i < batch.n; ++i) {
+      const BranchLayerTensors& t = layers[first + i];
+      batch.l[i] = StreamLayerPtrs{t.q, t.k_new, t.v_new, t.pk, t.pv, t.sk, t.sv, t.out, t.lse};
+    }
+    const BranchLayerTensors& t0 = layers[first];
+    cudaError_t e = launch_stream(t0.q, prefix, prefix_len, suffix, d_suffix_len, nullptr, max_suffix_len, n_branches,
+                                  q_heads, q_len, scale, t0.out, t0.lse, st, li, t0.k_new, t0.v_new, batch);
+    if (e != cudaSuccess) return e;
+  }
+  return cudaSuccess;
 }
 
 }  // namespace jup

@@ -115,6 +115,26 @@ cudaError_t launch_branch_tc(const bf16* q, const CacheView& prefix, int prefix_
 // status word like any kernel whose bounded wait ran out.
 cudaError_t launch_wait_probe(int* status, long long limit_cycles, cudaStream_t st, LaunchInfo& li);
 
+// The same step for several decoder layers in one launch of the streaming kernel (at most
+// kBranchMaxLayersPerLaunch per launch; more layers take further launches): every layer has its own tensors, all
+// share the geometry of `prefix` / `suffix` (whose own k / v are ignored), the lengths and the scale.
+constexpr int kBranchMaxLayersPerLaunch = 16;
+struct BranchLayerTensors {
+  const bf16* q;
+  const bf16* k_new;  // nullable (all layers alike): no fused KVCache write
+  const bf16* v_new;
+  const bf16* pk;
+  const bf16* pv;
+  const bf16* sk;
+  const bf16* sv;
+  float* out;
+  float* lse;  // nullable
+};
+cudaError_t launch_branch_stream_layers(const BranchLayerTensors* layers, int n_layers, const CacheView& prefix,
+                                        int prefix_len, const CacheView& suffix, const int32_t* d_suffix_len,
+                                        int max_suffix_len, int n_branches, int q_heads, int q_len, float scale,
+                                        cudaStream_t st, LaunchInfo& li);
+
 // Moves the accepted rows of every sequence's draft block (q_len <= 16 rows at d_pos[b]) to the front of the block.
 cudaError_t launch_kv_compact(const CacheView& c, int q_len, const int32_t* d_pos, const int32_t* d_accept,
                               const int32_t* d_n_accept, cudaStream_t st, LaunchInfo& li);
