@@ -542,7 +542,9 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
       constexpr int RPI = 32 / LPR;  // rows per warp iteration
       const int chunk = lane % LPR, sub = lane / LPR;
       const int x = warp >> 2;
-      const bool cta_ok = *abort_flag == 0;
+      // a CTA of the cluster that gave up on a wait has set the status word (before the barrier): its partials are
+      // incomplete, so nobody writes rows merged from them
+      const bool cta_ok = *abort_flag == 0 && *reinterpret_cast<volatile int*>(p.status) == 0;
       if (Tg[x] > 0) {  // the query tile exists
         // This lane finishes one 16-byte chunk of the rows (warp & 3) * 32 + it * RPI + sub, it = 0..LPR-1.
         // Loads go to L2 (the lines were written by other SMs) and are issued in batches before their first use.
@@ -673,7 +675,11 @@ static int max_resident_clusters() {
 }
 
 bool prefill_tc_supported(const CacheView& c, float scale) {
-  return c.head_dim == TC_D && scale > 0.f && scale < INFINITY && encode_fn() != nullptr;
+  // head_dim 128, a positive finite scale, and strides a tensor map can carry (multiples of 16 bytes below 2^40;
+  // the 16-byte rule is part of every cache descriptor already)
+  auto encodable = [](int64_t elems) { return static_cast<uint64_t>(elems) * 2 < (1ull << 40); };
+  return c.head_dim == TC_D && scale > 0.f && scale < INFINITY && encode_fn() != nullptr && encodable(c.sr) &&
+         encodable(c.sh) && encodable(c.sb);
 }
 
 // c: the attention's own segment (rows [0, pos + q_len) of every sequence); prefix (nullable): the segment in front
