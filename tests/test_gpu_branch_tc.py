@@ -127,6 +127,21 @@ def test_group_sizes_that_are_not_powers_of_two(ctx):
     run_case(ctx, 467, 4, 10, 2, 260, 3, [3, 128, 131, 40], "tree")         # group 5
 
 
+def test_random_geometry(ctx):
+    """Seeded random shapes: head counts and group sizes (powers of two or not), draft lengths, prefix and suffix lengths
+    around tile edges, few or many branches; every call mode."""
+    shapes = synth.uniform_ints(78, 1, 10 * 8, 0, 1 << 20).reshape(-1, 8)
+    for k, row in enumerate(shapes):
+        B = 1 + int(row[0]) % 20
+        Hkv = [1, 2, 4][int(row[1]) % 3]
+        G = [1, 2, 3, 4, 8][int(row[2]) % 5]
+        n = 1 + int(row[3]) % 16
+        P = [0, 1, 127, 128, 129, 500, 1100][int(row[4]) % 7]
+        lens = [n + int(x) % 420 for x in synth.uniform_ints(int(row[5]), 2, B, 0, 1 << 20)]
+        mode = ["plain", "fused", "tree"][k % 3]
+        run_case(ctx, 600 + k, B, Hkv * G, Hkv, P, n, lens, mode)
+
+
 def test_block_straddles_key_tiles(ctx):
     """The draft block crosses a 128-key tile edge: its rows are patched into two tiles."""
     for L in (129, 130, 131, 132, 256 + 2):
