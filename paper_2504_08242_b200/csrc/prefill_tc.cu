@@ -63,7 +63,11 @@ struct TcCfg {
   static constexpr int SOFTMAX_WARPS = 4 * NQ;
   static constexpr int LOADER_WARP = SOFTMAX_WARPS;
   static constexpr int MMA_WARP = SOFTMAX_WARPS + 1;
-  static constexpr int THREADS = 32 * (SOFTMAX_WARPS + 2);
+  // The two-warpgroup forms run three full warpgroups (the third: loader, MMA issuer, two idle warps) so that the
+  // register file can be re-divided: a softmax thread holds a whole score row (REGS_SOFTMAX), the third warpgroup
+  // gives its share back (REGS_OTHER); 2 x 128 x 208 + 128 x 88 = 384 x 168, the registers the CTA starts with.
+  static constexpr int THREADS = NQ == 2 ? 384 : 32 * (SOFTMAX_WARPS + 2);
+  static constexpr int REGS_SOFTMAX = 208, REGS_OTHER = 88;
   static constexpr int S_BUFS = NQ == 1 ? 2 : 1;  // S buffers per query tile
   static constexpr int O_COL0 = 256;
   // shared memory: [Q tiles][K ring][V ring][barriers]
@@ -87,7 +91,8 @@ enum {
   BAR_O_READY = 20,  // [2]
   BAR_DRAIN = 22,
   BAR_STORED = 23,   // the loader's cache stores have read their K/V slots
-  BAR_COUNT = 24
+  BAR_P_EARLY = 24,  // [2] the first 96 columns of P are in TMEM
+  BAR_COUNT = 26
 };
 
 constexpr int TC_BOX_FLOATS = TC_BM * 32;  // 16 KB
@@ -158,7 +163,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
 
   // ---- set-up
   if (threadIdx.x == 0) {
-    for (int i = 0; i < BAR_COUNT; ++i) mbar_init(bar(i), (i == BAR_P_FULL || i == BAR_P_FULL + 1) ? 128u : 1u);
+    for (int i = 0; i < BAR_COUNT; ++i) mbar_init(bar(i), (i == BAR_P_FULL || i == BAR_P_FULL + 1 || i == BAR_P_EARLY || i == BAR_P_EARLY + 1) ? 128u : 1u);
     *abort_flag = 0;
     mbar_fence_init();
   }
@@ -190,6 +195,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
 
   if (warp == Cfg::LOADER_WARP) {
     // =============================================================== loader
+    if constexpr (NQ == 2) reg_dec<Cfg::REGS_OTHER>();
     if (lane == 0) {
 #pragma unroll
       for (int x = 0; x < Cfg::Q_TILES; ++x) {
@@ -262,6 +268,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     __syncwarp();
   } else if (warp == Cfg::MMA_WARP) {
     // =============================================================== MMA issuer
+    if constexpr (NQ == 2) reg_dec<Cfg::REGS_OTHER>();
     if (lane == 0) {
       constexpr uint32_t idesc_qk = tc_idesc_bf16(TC_BM, TC_BN, false, false);
       constexpr uint32_t idesc_pv = tc_idesc_bf16(TC_BM, TC_D, false, true);
@@ -276,10 +283,11 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                     ks > 0);
         }
       };
-      auto issue_pv = [&](int x, int g, int buf, bool first) {  // O(x) (+)= P(x) V, V of load sequence number g
+      // O(x) (+)= P(x) V over the keys [16 ks0, 16 ks1) of the tile, V of load sequence number g
+      auto issue_pv = [&](int x, int g, int buf, bool first, int ks0, int ks1) {
         const uint32_t vb = sV + (g % KV_STAGES) * TC_TILE_BYTES;
 #pragma unroll
-        for (int ks = 0; ks < TC_BN / 16; ++ks)
+        for (int ks = ks0; ks < ks1; ++ks)
           tc_mma_ts(o_col(x), s_col(x, buf) + ks * 8, tc_smem_desc(vb + ks * 2048, TC_PANEL_BYTES, 1024), idesc_pv,
                     (!first || ks > 0));
       };
@@ -334,10 +342,14 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
             tc_commit(bar(BAR_K_EMPTY + gn % KV_STAGES));
           }
           need_v(g);
+          ok = ok && mbar_wait(bar(BAR_P_EARLY + x), j & 1, abort_flag, p.status);
+          if (!ok) break;
+          tc_fence_after();
+          issue_pv(x, g, buf, j == 0, 0, 6);  // the first 96 keys while the softmax finishes the last 32
           ok = ok && mbar_wait(bar(BAR_P_FULL + x), j & 1, abort_flag, p.status);
           if (!ok) break;
           tc_fence_after();
-          issue_pv(x, g, buf, j == 0);
+          issue_pv(x, g, buf, j == 0, 6, 8);
           tc_commit(bar(BAR_O_READY + x));
           if (x == last_user(g)) tc_commit(bar(BAR_V_EMPTY + g % KV_STAGES));
           if (NQ == 2 && j + 1 < T[x]) {
@@ -356,8 +368,9 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
       }
     }
     __syncwarp();
-  } else {
+  } else if (warp < Cfg::SOFTMAX_WARPS) {
     // =============================================================== softmax warpgroups
+    if constexpr (NQ == 2) reg_inc<Cfg::REGS_SOFTMAX>();
     const int x = warp >> 2;                      // query tile (key-split mode: stream) of this warpgroup
     const int row_in_tile = (warp & 3) * 32 + lane;
     const int row = (SPLIT ? qblk : qblk * NQ + x) * TC_BM + row_in_tile;  // row inside the chunk
@@ -381,9 +394,15 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
       const int nvalid = g < Tp ? p.prefix_len - g * TC_BN : lim - (g - Tp) * TC_BN;
       // warp-uniform flag, so the warp stays converged for the collective tcgen05 operations
       const bool masked = __any_sync(0xffffffffu, nvalid < TC_BN);
-      ok = softmax_tile_step<PARTIAL>(tS, tO, j, masked, ColumnLimit{nvalid}, c, m_ref, l, [&] {
-        return mbar_wait(bar(BAR_O_READY + x), (j - 1) & 1, abort_flag, p.status);
-      });
+      // (the accumulator's barrier is only consulted when O has to be rescaled: phase j - 1 cannot be overtaken,
+      // because PV(j) needs this thread's P(j))
+      ok = softmax_tile_row<PARTIAL>(
+          tS, tO, j, masked, ColumnLimit{nvalid}, c, m_ref, l,
+          [&] { return mbar_wait(bar(BAR_O_READY + x), (j - 1) & 1, abort_flag, p.status); },
+          [&] {
+            tc_fence_before();
+            mbar_arrive(bar(BAR_P_EARLY + x));
+          });
       if (!ok) break;
       tc_fence_before();
       mbar_arrive(bar(BAR_P_FULL + x));
@@ -490,6 +509,10 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         p.lse[(static_cast<int64_t>(b) * p.q_heads + h) * p.q_len + row] =
             (m_ref + log2f(l)) * 0.69314718055994530942f;
     }
+  }
+
+  else if constexpr (NQ == 2) {
+    reg_dec<Cfg::REGS_OTHER>();  // the idle warps of the third warpgroup: the re-division is a warpgroup's decision
   }
 
   if constexpr (CL > 1) {

@@ -140,6 +140,98 @@ __device__ __forceinline__ bool softmax_tile_step(uint32_t tS, uint32_t tO, int 
   return true;
 }
 
+// The same step with the whole score row in registers (needs about 200 registers per thread): one load of the 128
+// scores, the row maximum, at most one move of the reference per tile (decided before any P is written, so no P
+// chunk is ever corrected), then P in four chunks of 32 columns.  After the third chunk is in TMEM (tcgen05.wait::st
+// done) release_early() runs: the caller signals the MMA issuer, which starts O += P V on the first 96 keys while
+// this thread still computes the last 32.  wait_o() is only called when the accumulator has to be rescaled
+// (j > 0); it waits until O(j-1) is complete and returns false if the wait gave up, and then so does this function.
+// On return P is complete in TMEM; the caller fences and signals the second half.
+template <bool PARTIAL, class Allow, class WaitO, class Release>
+__device__ __forceinline__ bool softmax_tile_row(uint32_t tS, uint32_t tO, int j, bool masked, const Allow& allow, float c,
+                                                 float& m_ref, float& l, WaitO&& wait_o, Release&& release_early) {
+  uint32_t sv[128];
+#pragma unroll
+  for (int q4 = 0; q4 < 4; ++q4) tmem_ld32(tS + q4 * 32, *reinterpret_cast<uint32_t(*)[32]>(&sv[q4 * 32]));
+  tc_wait_ld();
+  if (masked) {
+#pragma unroll
+    for (int i = 0; i < 128; ++i)
+      if (!allow(i)) sv[i] = 0xff800000u;  // -inf
+  }
+  // ---- row maximum: 3-input max, 32 + 8 + 8 + 3 + 3 + 1 operations in chains of depth 5
+  float mx;
+  {
+    float a[32];
+#pragma unroll
+    for (int k = 0; k < 32; ++k)
+      a[k] = fmax3(__uint_as_float(sv[4 * k]), __uint_as_float(sv[4 * k + 1]), __uint_as_float(sv[4 * k + 2]));
+    float b[8], d[8];
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+      b[k] = fmax3(fmax3(a[4 * k], a[4 * k + 1], a[4 * k + 2]), a[4 * k + 3], __uint_as_float(sv[16 * k + 3]));
+      d[k] = fmax3(__uint_as_float(sv[16 * k + 7]), __uint_as_float(sv[16 * k + 11]), __uint_as_float(sv[16 * k + 15]));
+    }
+    mx = fmaxf(fmax3(fmax3(b[0], b[1], b[2]), fmax3(b[3], b[4], b[5]), fmaxf(b[6], b[7])),
+               fmax3(fmax3(d[0], d[1], d[2]), fmax3(d[3], d[4], d[5]), fmaxf(d[6], d[7])));
+  }
+  const float mxs = mx * c;
+  // lazy reference: it only moves when the maximum outgrew it by 2^8 (a row that has seen nothing keeps -inf,
+  // and its first visible score moves it because -inf + 8 is still -inf)
+  const bool grow = mxs > m_ref + TC_RESCALE_THRESHOLD;
+  if (__any_sync(0xffffffffu, grow)) {
+    const float alpha = grow ? fast_exp2(m_ref - mxs) : 1.f;
+    l *= alpha;
+    if (grow) m_ref = mxs;
+    if (j > 0) {  // O(j-1) must be complete before it is rescaled
+      if (!wait_o()) return false;
+      tc_fence_after();
+#pragma unroll
+      for (int q4 = 0; q4 < 4; ++q4) {
+        uint32_t o[32];
+        tmem_ld32(tO + q4 * 32, o);
+        tc_wait_ld();
+#pragma unroll
+        for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
+        tmem_st32(tO + q4 * 32, o);
+      }
+    }
+  }
+  // ---- P
+  const float nm = (PARTIAL && m_ref == -INFINITY) ? 0.f : -m_ref;
+  const uint64_t nm2 = pack2(nm, nm), c2 = pack2(c, c);
+  uint64_t lacc[4];
+#pragma unroll
+  for (int k = 0; k < 4; ++k) lacc[k] = pack2(0.f, 0.f);
+#pragma unroll
+  for (int q4 = 0; q4 < 4; ++q4) {
+    uint32_t pk[16];
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+      const uint64_t x =
+          fma2(pack2(__uint_as_float(sv[q4 * 32 + 2 * i]), __uint_as_float(sv[q4 * 32 + 2 * i + 1])), c2, nm2);
+      float x0, x1;
+      unpack2(x, x0, x1);
+      const float p0 = fast_exp2(x0), p1 = fast_exp2(x1);
+      lacc[i & 3] = add2(lacc[i & 3], pack2(p0, p1));
+      pk[i] = pack_bf16(p0, p1);
+    }
+    tmem_st16(tS + q4 * 16, pk);
+    if (q4 == 2) {
+      tc_wait_st();
+      release_early();
+    }
+  }
+  {
+    float a0, a1, b0, b1;
+    unpack2(add2(lacc[0], lacc[1]), a0, a1);
+    unpack2(add2(lacc[2], lacc[3]), b0, b1);
+    l += (a0 + a1) + (b0 + b1);
+  }
+  tc_wait_st();
+  return true;
+}
+
 // Output staging for a tiled store: a box of 128 rows x 32 fp32 (128-byte rows, 16-byte chunks XOR-swizzled by
 // the row as the 128-byte swizzle of the tensor map expects; conflict-free for one thread per row).
 __device__ __forceinline__ void stage_box_row(float* box, int r, const float (&v)[32]) {
