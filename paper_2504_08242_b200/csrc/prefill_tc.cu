@@ -274,22 +274,26 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
       constexpr uint32_t idesc_pv = tc_idesc_bf16(TC_BM, TC_D, false, true);
       auto s_col = [&](int x, int buf) { return tmem + (NQ == 2 ? x * 128 : buf * 128); };
       auto o_col = [&](int x) { return tmem + Cfg::O_COL0 + x * 128; };
+      // The issue loops are kept to an integer addition or two per MMA (descriptor halves, see tc_desc_lo): this
+      // thread shares its scheduler with two softmax warps, and a longer chain of address arithmetic per MMA
+      // made the issue, not the tensor pipe, the limit.
       auto issue_qk = [&](int x, int g, int buf) {  // S(x) = Q(x) K^T, K of load sequence number g
-        const uint32_t qb = sQ + (SPLIT ? 0 : x) * TC_TILE_BYTES, kb = sK + (g % KV_STAGES) * TC_TILE_BYTES;
+        const uint32_t q_lo = tc_desc_lo(sQ + (SPLIT ? 0 : x) * TC_TILE_BYTES, 16);
+        const uint32_t k_lo = tc_desc_lo(sK + (g % KV_STAGES) * TC_TILE_BYTES, 16);
+        const uint32_t d = s_col(x, buf);
 #pragma unroll
         for (int ks = 0; ks < TC_D / 16; ++ks) {
-          const uint32_t off = (ks >> 2) * TC_PANEL_BYTES + (ks & 3) * 32;
-          tc_mma_ss(s_col(x, buf), tc_smem_desc(qb + off, 16, 1024), tc_smem_desc(kb + off, 16, 1024), idesc_qk,
-                    ks > 0);
+          const uint32_t off = ((ks >> 2) * TC_PANEL_BYTES + (ks & 3) * 32) >> 4;
+          tc_mma_ss_lo(d, q_lo + off, k_lo + off, idesc_qk, ks > 0);
         }
       };
       // O(x) (+)= P(x) V over the keys [16 ks0, 16 ks1) of the tile, V of load sequence number g
       auto issue_pv = [&](int x, int g, int buf, bool first, int ks0, int ks1) {
-        const uint32_t vb = sV + (g % KV_STAGES) * TC_TILE_BYTES;
+        const uint32_t v_lo = tc_desc_lo(sV + (g % KV_STAGES) * TC_TILE_BYTES, TC_PANEL_BYTES);
+        const uint32_t d = o_col(x), a = s_col(x, buf);
 #pragma unroll
         for (int ks = ks0; ks < ks1; ++ks)
-          tc_mma_ts(o_col(x), s_col(x, buf) + ks * 8, tc_smem_desc(vb + ks * 2048, TC_PANEL_BYTES, 1024), idesc_pv,
-                    (!first || ks > 0));
+          tc_mma_ts_lo(d, a + ks * 8, v_lo + ks * (2048 >> 4), idesc_pv, (!first || ks > 0));
       };
       auto last_user = [&](int g) {  // the last stream (in issue order) that uses the tile of sequence number g
         if (SPLIT) return g & 1;
