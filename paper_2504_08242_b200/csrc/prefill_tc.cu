@@ -645,7 +645,30 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
   }
 }
 
+}  // namespace jup
+
+#include "prefill_tc_frag.cuh"
+
+namespace jup {
+
 // ---------------------------------------------------------------- host side
+
+static cudaError_t launch_frag(int64_t ctas, cudaStream_t st, const CUtensorMap& tq, const CUtensorMap& tk,
+                               const CUtensorMap& tv, const CUtensorMap& tpk, const CUtensorMap& tpv,
+                               const CUtensorMap& tck, const CUtensorMap& tcv, const TcParams& p) {
+  static PerDeviceOnce done;
+  if (!done.done()) {
+    cudaError_t e =
+        cudaFuncSetAttribute(prefill_frag_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, FragCfg::SMEM_BYTES);
+    if (e == cudaSuccess)
+      e = cudaFuncSetAttribute(prefill_frag_kernel, cudaFuncAttributePreferredSharedMemoryCarveout,
+                               cudaSharedmemCarveoutMaxShared);
+    if (e != cudaSuccess) return e;
+    done.set();
+  }
+  return launch_pdl_cluster(prefill_frag_kernel, dim3(static_cast<unsigned>(ctas)), dim3(FragCfg::THREADS),
+                            FragCfg::SMEM_BYTES, st, 1u, tq, tk, tv, tpk, tpv, tck, tcv, p);
+}
 
 template <int NQ, bool SPLIT, int CL>
 static cudaError_t launch_variant(int64_t ctas, cudaStream_t st, const CUtensorMap& tq, const CUtensorMap& tk,
@@ -807,12 +830,9 @@ static cudaError_t launch_tc(const bf16* q, const CacheView& c, const CacheView*
   } else if (cl == 4) {
     p.q_blocks = (q_len + 255) / 256;
     e = launch_variant<2, false, 4>(ctas2, st, tq, tk, tv, tpk, tpv, to, tck, tcv, p);
-  } else if (ctas1 <= li.sm_count) {
-    p.q_blocks = (q_len + 127) / 128;
-    e = launch_variant<2, true, 1>(ctas1, st, tq, tk, tv, tpk, tpv, to, tck, tcv, p);
   } else {
     p.q_blocks = (q_len + 127) / 128;
-    e = launch_variant<1, false, 1>(ctas1, st, tq, tk, tv, tpk, tpv, to, tck, tcv, p);
+    e = launch_frag(ctas1, st, tq, tk, tv, tpk, tpv, tck, tcv, p);
   }
   li.launches += 1;
   return e;

@@ -232,6 +232,127 @@ __device__ __forceinline__ bool softmax_tile_row(uint32_t tS, uint32_t tO, int j
   return true;
 }
 
+// ---------------------------------------------------------------- fragment form
+// A warp owns 16 query rows of the tile (TMEM lanes lane0 .. lane0 + 15, tS / tO carry that lane) and holds their
+// 128 scores in the 16x256b layout: thread t has rows A = t/4 and B = 8 + t/4, columns 8k + 2 (t mod 4) + {0, 1},
+// k = 0..15 -- 64 scores per thread, half of what a thread-per-row layout holds, so two warpgroups can share one
+// tile (each taking 16 of every 32 rows) and a tile's softmax takes half as long.  Row maxima are completed over
+// the four threads of a row with two shuffles; the reference m_ref[e] is the same in the four threads, l[e] is a
+// per-thread partial sum (added up over the quad after the walk).  Otherwise as softmax_tile_row: lazy reference,
+// at most one move per tile, P written as bf16 pairs over the S columns, released in two parts.
+// allow(e, col): row e (0: A, 1: B) sees column col; only consulted when masked (warp-uniform).
+__device__ __forceinline__ float max32_strided(const uint32_t (&sv)[64], int e) {
+  // the 32 values of row e: sv[4k + 2e], sv[4k + 2e + 1]
+  float a[11];
+#pragma unroll
+  for (int i = 0; i < 10; ++i) {
+    const int v0 = 3 * i, v1 = 3 * i + 1, v2 = 3 * i + 2;  // value indices 0..31 -> register 4 (v / 2) + 2 e + (v & 1)
+    a[i] = fmax3(__uint_as_float(sv[4 * (v0 >> 1) + 2 * e + (v0 & 1)]), __uint_as_float(sv[4 * (v1 >> 1) + 2 * e + (v1 & 1)]),
+                 __uint_as_float(sv[4 * (v2 >> 1) + 2 * e + (v2 & 1)]));
+  }
+  a[10] = fmaxf(__uint_as_float(sv[4 * 15 + 2 * e]), __uint_as_float(sv[4 * 15 + 2 * e + 1]));
+  const float b0 = fmax3(a[0], a[1], a[2]), b1 = fmax3(a[3], a[4], a[5]), b2 = fmax3(a[6], a[7], a[8]);
+  return fmax3(fmax3(b0, b1, b2), a[9], a[10]);
+}
+
+// The step in pieces, so that a kernel can run the pieces of consecutive tiles against each other (scores of tile
+// j + 1 loaded and reduced to their row maxima while the exponentials of tile j keep the special-function unit busy).
+
+// Row maxima (times c, over the four threads of each row) of a tile held in fragments; masks hidden columns first.
+template <class Allow>
+__device__ __forceinline__ void frag_mask_max(uint32_t (&sv)[64], bool masked, const Allow& allow, int col0, float c,
+                                              float (&mxs)[2]) {
+  if (masked) {
+#pragma unroll
+    for (int k = 0; k < 16; ++k)
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+        if (!allow(i >> 1, 8 * k + col0 + (i & 1))) sv[4 * k + i] = 0xff800000u;  // -inf
+  }
+#pragma unroll
+  for (int e = 0; e < 2; ++e) {
+    float mx = max32_strided(sv, e);
+    mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+    mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+    mxs[e] = mx * c;
+  }
+}
+
+// Lazy reference: moves m_ref[e] to the tile's maximum when that outgrew it by 2^8 and scales l and, from the second
+// tile on, the accumulator rows (wait_o(): bounded wait until O holds the tiles before this one; false: gave up).
+template <class WaitO>
+__device__ __forceinline__ bool frag_decide(const float (&mxs)[2], float (&m_ref)[2], float (&l)[2], uint32_t tO, int j,
+                                            WaitO&& wait_o) {
+  bool grow[2];
+#pragma unroll
+  for (int e = 0; e < 2; ++e) grow[e] = mxs[e] > m_ref[e] + TC_RESCALE_THRESHOLD;
+  if (__any_sync(0xffffffffu, grow[0] || grow[1])) {
+    float alpha[2];
+#pragma unroll
+    for (int e = 0; e < 2; ++e) {
+      alpha[e] = grow[e] ? fast_exp2(m_ref[e] - mxs[e]) : 1.f;
+      l[e] *= alpha[e];
+      if (grow[e]) m_ref[e] = mxs[e];
+    }
+    if (j > 0) {
+      if (!wait_o()) return false;
+      tc_fence_after();
+#pragma unroll
+      for (int hh = 0; hh < 2; ++hh) {
+        uint32_t o[32];
+        tmem_ld_16x256b_x8(tO + hh * 64, o);
+        tc_wait_ld();
+#pragma unroll
+        for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha[(i >> 1) & 1]);
+        tmem_st_16x256b_x8(tO + hh * 64, o);
+      }
+    }
+  }
+  return true;
+}
+
+// P = exp2(s c - m_ref) as bf16 pairs over the first 64 columns of the tile's S buffer, row sums into l; mid() runs
+// after the first half (the caller's work on the next tile goes there).  Returns with the stores issued, not waited.
+template <class Mid>
+__device__ __forceinline__ void frag_exp_store(const uint32_t (&sv)[64], uint32_t tS, float c, const float (&m_ref)[2],
+                                               float (&l)[2], Mid&& mid) {
+  uint64_t nm2[2];
+#pragma unroll
+  for (int e = 0; e < 2; ++e) {
+    const float nm = m_ref[e] == -INFINITY ? 0.f : -m_ref[e];
+    nm2[e] = pack2(nm, nm);
+  }
+  const uint64_t c2 = pack2(c, c);
+  uint64_t lacc[2][2];
+#pragma unroll
+  for (int e = 0; e < 2; ++e) lacc[e][0] = lacc[e][1] = pack2(0.f, 0.f);
+  uint32_t w[32];  // P: w[2k + e] = keys 8k + col0 + {0, 1} of row e
+#pragma unroll
+  for (int k = 0; k < 16; ++k) {
+#pragma unroll
+    for (int e = 0; e < 2; ++e) {
+      const uint64_t x =
+          fma2(pack2(__uint_as_float(sv[4 * k + 2 * e]), __uint_as_float(sv[4 * k + 2 * e + 1])), c2, nm2[e]);
+      float x0, x1;
+      unpack2(x, x0, x1);
+      const float p0 = fast_exp2(x0), p1 = fast_exp2(x1);
+      lacc[e][k & 1] = add2(lacc[e][k & 1], pack2(p0, p1));
+      w[2 * k + e] = pack_bf16(p0, p1);
+    }
+    if (k == 7) {
+      tmem_st_16x128b_x8(tS, &w[0]);
+      mid();
+    }
+  }
+  tmem_st_16x128b_x8(tS + 32, &w[16]);
+#pragma unroll
+  for (int e = 0; e < 2; ++e) {
+    float a0, a1;
+    unpack2(add2(lacc[e][0], lacc[e][1]), a0, a1);
+    l[e] += a0 + a1;
+  }
+}
+
 // Output staging for a tiled store: a box of 128 rows x 32 fp32 (128-byte rows, 16-byte chunks XOR-swizzled by
 // the row as the 128-byte swizzle of the tensor map expects; conflict-free for one thread per row).
 __device__ __forceinline__ void stage_box_row(float* box, int r, const float (&v)[32]) {
