@@ -22,7 +22,7 @@ struct FragCfg {
   static constexpr int STAGES = 3;  // K slots = V slots = S buffers
   static constexpr int SOFTMAX_WARPS = 8, LOADER_WARP = 8, MMA_WARP = 9, WATCH_WARP = 10;
   static constexpr int THREADS = 384;
-  static constexpr int REGS_SOFTMAX = 208, REGS_OTHER = 88;  // 2 x 128 x 208 + 128 x 88 = 384 x 168
+  static constexpr int REGS_SOFTMAX = 216, REGS_OTHER = 72;  // 2 x 128 x 216 + 128 x 72 = 384 x 168
   static constexpr int O_COL0 = 384;
   static constexpr int SMEM_Q = 0;
   static constexpr int SMEM_K = TC_TILE_BYTES;
@@ -246,7 +246,7 @@ prefill_frag_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       for (int j = 0; j < T && ok; ++j) {
         ok = landed(FB_V_FULL, j);
         if (ok && j + STAGES < T) ok = landed(FB_K_FULL, j + STAGES);
-        ok = ok && mbar_wait(bar3(FB_P_FULL, j), par3(j), abort_flag, p.status);
+        ok = ok && mbar_spin_wait(bar3(FB_P_FULL, j), par3(j), abort_flag, p.status);
         if (!ok) break;
         count_publish(go_count, ++step);
       }
@@ -274,52 +274,60 @@ prefill_frag_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
       if (j + 2 < T) return mbar_wait(bar3(FB_S_FULL, j + 2), par3(j + 2), abort_flag, p.status);
       return mbar_wait(bar(FB_O_READY + j - 1 - o0), 0, abort_flag, p.status);
     };
-    // scores of tile j: fetch into fragments, mask, row maxima.  Columns >= nvalid are hidden: the end of the front
-    // segment in its last tile, the causal limit afterwards.
+    // Scores of tile j into fragments (asynchronous: the registers may only be used after the load was waited for).
     auto fetch = [&](int j, uint32_t (&sv)[64]) {
-      ok = mbar_wait(bar3(FB_S_FULL, j), par3(j), abort_flag, p.status);
+      ok = mbar_spin_wait(bar3(FB_S_FULL, j), par3(j), abort_flag, p.status);
       if (!ok) return;
       tc_fence_after();
       tmem_ld_16x256b_x16(taddr + (j % STAGES) * 128, sv);
     };
-    auto reduce = [&](int j, uint32_t (&sv)[64]) {
-      int nvalid[2];
+    // Columns >= nvalid of a row are hidden: the end of the front segment in its last tile, the causal limit afterwards.
+    int nvalid[2];
+    auto tile_masked = [&](int j) {  // warp-uniform; fills nvalid
 #pragma unroll
       for (int e = 0; e < 2; ++e) nvalid[e] = j < Tp ? p.prefix_len - j * TC_BN : lim[e] - (j - Tp) * TC_BN;
-      const bool masked = __any_sync(0xffffffffu, nvalid[0] < TC_BN || nvalid[1] < TC_BN);
-      frag_mask_max(sv, masked, [&](int e, int col) { return col < nvalid[e]; }, col0, c, mxs);
+      return __any_sync(0xffffffffu, nvalid[0] < TC_BN || nvalid[1] < TC_BN) != 0;
     };
-    // one tile: cur holds its masked scores and mxs its maxima; the next tile's go into nxt meanwhile
+    auto apply_mask = [&](uint32_t (&sv)[64]) {
+#pragma unroll
+      for (int k = 0; k < 16; ++k)
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+          if (8 * k + col0 + (i & 1) >= nvalid[i >> 1]) sv[4 * k + i] = 0xff800000u;  // -inf
+    };
+    // One tile: cur holds its masked scores and mxs its maxima; nxt is the next tile's fetch in flight, whose maxima
+    // are worked out between this tile's exponentials; afterwards the fetch of the tile after that goes into cur.
     auto tile = [&](int j, uint32_t (&cur)[64], uint32_t (&nxt)[64]) {
       if (!frag_decide(mxs, m_ref, l, tO, j, [&] { return wait_o_before(j); })) {
         ok = false;
         return;
       }
-      // the next tile's scores are fetched half-way through this tile's exponentials and waited for at once: the
-      // registers of a fetch in flight must not be live across other code (the compiler may move or spill them)
-      frag_exp_store(cur, taddr + (j % STAGES) * 128, c, m_ref, l, [&] {
-        if (j + 1 < T) {
-          fetch(j + 1, nxt);
-          tc_wait_ld();
-          if (ok) reduce(j + 1, nxt);
-        }
-      });
-      if (!ok) return;
+      const bool next_masked = j + 1 < T && tile_masked(j + 1);
+      float mxs_next[2];
+      frag_exp_store_max(cur, taddr + (j % STAGES) * 128, c, m_ref, l, nxt, next_masked, [&] { apply_mask(nxt); }, mxs_next);
+      mxs[0] = mxs_next[0];
+      mxs[1] = mxs_next[1];
       tc_wait_st();
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(bar3(FB_P_FULL, j));
+      if (j + 2 < T) fetch(j + 2, cur);
     };
     uint32_t fa[64], fb[64];
+#pragma unroll
+    for (int i = 0; i < 64; ++i) fb[i] = 0u;  // read (and ignored) as "next tile" when there is none
     fetch(0, fa);
     if (ok) {
-      tc_wait_ld();
-      reduce(0, fa);
+      tc_wait_ld_into(fa);
+      const bool masked0 = tile_masked(0);
+      frag_mask_max(fa, masked0, [&](int e, int col) { return col < nvalid[e]; }, col0, c, mxs);
+      if (T > 1) fetch(1, fb);
     }
     for (int j = 0; j < T && ok; j += 2) {
       tile(j, fa, fb);
       if (j + 1 < T && ok) tile(j + 1, fb, fa);
     }
+    tc_wait_ld();  // (no fetch is left in flight; the registers are dead)
     pdl_launch_dependents();  // the next kernel of the stream may start its own set-up now
     ok = ok && mbar_wait(bar(FB_O_READY + T - 1 - o0), 0, abort_flag, p.status);  // the accumulator is final
     tc_fence_after();

@@ -353,6 +353,74 @@ __device__ __forceinline__ void frag_exp_store(const uint32_t (&sv)[64], uint32_
   }
 }
 
+// The same with the next tile's row maxima worked in: nxt is a fragment load in flight (or stale registers when there
+// is no next tile; the result is then unused).  It is waited for after the fourth of the sixteen steps, masked if
+// need be (mask_next(), warp-uniform and rare), and its 2 x 32 values are folded into running maxima a few per step,
+// so that their arithmetic issues in the gaps of the exponentials instead of after them.  mxs_next: maxima times c.
+template <class MaskNext>
+__device__ __forceinline__ void frag_exp_store_max(const uint32_t (&sv)[64], uint32_t tS, float c, const float (&m_ref)[2],
+                                                   float (&l)[2], uint32_t (&nxt)[64], bool next_masked,
+                                                   MaskNext&& mask_next, float (&mxs_next)[2]) {
+  uint64_t nm2[2];
+#pragma unroll
+  for (int e = 0; e < 2; ++e) {
+    const float nm = m_ref[e] == -INFINITY ? 0.f : -m_ref[e];
+    nm2[e] = pack2(nm, nm);
+  }
+  const uint64_t c2 = pack2(c, c);
+  uint64_t lacc[2][2];
+#pragma unroll
+  for (int e = 0; e < 2; ++e) lacc[e][0] = lacc[e][1] = pack2(0.f, 0.f);
+  float ma[2][2] = {{-INFINITY, -INFINITY}, {-INFINITY, -INFINITY}};  // running maxima of the next tile, two chains per row
+  uint32_t w[32];  // P: w[2k + e] = keys 8k + col0 + {0, 1} of row e
+#pragma unroll
+  for (int k = 0; k < 16; ++k) {
+#pragma unroll
+    for (int e = 0; e < 2; ++e) {
+      const uint64_t x =
+          fma2(pack2(__uint_as_float(sv[4 * k + 2 * e]), __uint_as_float(sv[4 * k + 2 * e + 1])), c2, nm2[e]);
+      float x0, x1;
+      unpack2(x, x0, x1);
+      const float p0 = fast_exp2(x0), p1 = fast_exp2(x1);
+      lacc[e][k & 1] = add2(lacc[e][k & 1], pack2(p0, p1));
+      w[2 * k + e] = pack_bf16(p0, p1);
+    }
+    if (k == 3) {
+      tc_wait_ld_into(nxt);
+      if (next_masked) mask_next();
+    }
+    if (k >= 4 && k < 12) {  // two of the next tile's sixteen column blocks per step
+#pragma unroll
+      for (int kk = 2 * (k - 4); kk < 2 * (k - 4) + 2; ++kk)
+#pragma unroll
+        for (int e = 0; e < 2; ++e)
+          ma[e][kk & 1] = fmax3(ma[e][kk & 1], __uint_as_float(nxt[4 * kk + 2 * e]), __uint_as_float(nxt[4 * kk + 2 * e + 1]));
+    }
+    if (k == 7) tmem_st_16x128b_x8(tS, &w[0]);
+    if (k == 12) {
+#pragma unroll
+      for (int e = 0; e < 2; ++e) {
+        ma[e][0] = fmaxf(ma[e][0], ma[e][1]);
+        ma[e][0] = fmaxf(ma[e][0], __shfl_xor_sync(0xffffffffu, ma[e][0], 1));
+      }
+    }
+    if (k == 14) {
+#pragma unroll
+      for (int e = 0; e < 2; ++e) {
+        ma[e][0] = fmaxf(ma[e][0], __shfl_xor_sync(0xffffffffu, ma[e][0], 2));
+        mxs_next[e] = ma[e][0] * c;
+      }
+    }
+  }
+  tmem_st_16x128b_x8(tS + 32, &w[16]);
+#pragma unroll
+  for (int e = 0; e < 2; ++e) {
+    float a0, a1;
+    unpack2(add2(lacc[e][0], lacc[e][1]), a0, a1);
+    l[e] += a0 + a1;
+  }
+}
+
 // Output staging for a tiled store: a box of 128 rows x 32 fp32 (128-byte rows, 16-byte chunks XOR-swizzled by
 // the row as the 128-byte swizzle of the tensor map expects; conflict-free for one thread per row).
 __device__ __forceinline__ void stage_box_row(float* box, int r, const float (&v)[32]) {
