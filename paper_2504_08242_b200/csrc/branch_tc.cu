@@ -374,20 +374,21 @@ branch_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
       constexpr uint32_t idesc_qk = tc_idesc_bf16(BT_BM, BT_BN, false, false);
       constexpr uint32_t idesc_pv = tc_idesc_bf16(BT_BM, BT_D, false, true);
       const uint32_t s_col = tmem + x * 128, o_col = tmem + 256 + x * 128;
+      // descriptor halves (tc_desc_lo): one integer addition per operand slice keeps the issue loop short
+      const uint32_t q_lo = tc_desc_lo(sQ, 16);
       auto issue_qk = [&](int s) {  // S = Q K^T, K of sequence number s
-        const uint32_t kb = sK + (s % KV_STAGES) * BT_TILE_BYTES;
+        const uint32_t k_lo = tc_desc_lo(sK + (s % KV_STAGES) * BT_TILE_BYTES, 16);
 #pragma unroll
         for (int ks = 0; ks < BT_D / 16; ++ks) {
-          const uint32_t off = (ks >> 2) * BT_PANEL_BYTES + (ks & 3) * 32;
-          tc_mma_ss(s_col, tc_smem_desc(sQ + off, 16, 1024), tc_smem_desc(kb + off, 16, 1024), idesc_qk, ks > 0);
+          const uint32_t off = ((ks >> 2) * BT_PANEL_BYTES + (ks & 3) * 32) >> 4;
+          tc_mma_ss_lo(s_col, q_lo + off, k_lo + off, idesc_qk, ks > 0);
         }
       };
       auto issue_pv = [&](int s, bool first) {  // O (+)= P V, V of sequence number s
-        const uint32_t vb = sV + (s % KV_STAGES) * BT_TILE_BYTES;
+        const uint32_t v_lo = tc_desc_lo(sV + (s % KV_STAGES) * BT_TILE_BYTES, BT_PANEL_BYTES);
 #pragma unroll
         for (int ks = 0; ks < BT_BN / 16; ++ks)
-          tc_mma_ts(o_col, s_col + ks * 8, tc_smem_desc(vb + ks * 2048, BT_PANEL_BYTES, 1024), idesc_pv,
-                    (!first || ks > 0));
+          tc_mma_ts_lo(o_col, s_col + ks * 8, v_lo + ks * (2048 >> 4), idesc_pv, (!first || ks > 0));
       };
       bool ok = mbar_wait(bar(BT_Q_FULL), 0, abort_flag, p.status, wl);  // (also when the list is empty: the copy must land)
       auto need_k = [&](int s) {

@@ -381,6 +381,28 @@ __device__ __forceinline__ float fmax3(float a, float b, float c) {
   asm("max.f32 %0, %1, %2, %3;\n" : "=f"(r) : "f"(a), "f"(b), "f"(c));
   return r;
 }
+// 2^x for a packed pair on the FMA pipe instead of the special-function unit (which is the softmax's bottleneck:
+// 16 results per clock per SM against 128 FMAs): x = n + f with n the nearest integer (magic-number rounding) and f
+// in [-0.5, 0.5], a degree-3 polynomial for 2^f (relative error 7.5e-5, far below the bf16 rounding P gets anyway),
+// n added into the exponent field.  Inputs below -126 (masked scores are -inf) give 2^-126.
+__device__ __forceinline__ uint64_t exp2_poly_pair(uint64_t x) {
+  float x0, x1;
+  unpack2(x, x0, x1);
+  const uint64_t xc = pack2(fmaxf(x0, -126.f), fmaxf(x1, -126.f));
+  const uint64_t t = add2(xc, pack2(12582912.f, 12582912.f));        // 1.5 * 2^23: the integer lands in the low bits
+  const uint64_t n = add2(t, pack2(-12582912.f, -12582912.f));
+  const uint64_t f = fma2(n, pack2(-1.f, -1.f), xc);
+  uint64_t p = fma2(pack2(0.0551716648f, 0.0551716648f), f, pack2(0.2426111251f, 0.2426111251f));
+  p = fma2(p, f, pack2(0.6932609677f, 0.6932609677f));
+  p = fma2(p, f, pack2(0.9999280572f, 0.9999280572f));
+  float p0, p1, t0, t1;
+  unpack2(p, p0, p1);
+  unpack2(t, t0, t1);
+  const float r0 = __int_as_float(__float_as_int(p0) + (__float_as_int(t0) << 23));
+  const float r1 = __int_as_float(__float_as_int(p1) + (__float_as_int(t1) << 23));
+  return pack2(r0, r1);
+}
+
 template <int N>
 __device__ __forceinline__ void reg_inc() {
   asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;\n" ::"n"(N));

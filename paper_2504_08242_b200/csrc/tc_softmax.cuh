@@ -353,6 +353,14 @@ __device__ __forceinline__ void frag_exp_store(const uint32_t (&sv)[64], uint32_
   }
 }
 
+// Which of a tile's 32 column pairs per thread (step k, row e) take their exponentials on the FMA pipe.
+#ifndef JUP_EXP_EMU
+#define JUP_EXP_EMU 1
+#endif
+__device__ __forceinline__ constexpr bool frag_exp_on_fma(int k, int e) {
+  return JUP_EXP_EMU == 1 ? (e == 1 && (k & 1)) : JUP_EXP_EMU == 2 ? (e == 1) : JUP_EXP_EMU == 3 ? (e == 1 && (k & 3) == 3) : false;
+}
+
 // The same with the next tile's row maxima worked in: nxt is a fragment load in flight (or stale registers when there
 // is no next tile; the result is then unused).  It is waited for after the fourth of the sixteen steps, masked if
 // need be (mask_next(), warp-uniform and rare), and its 2 x 32 values are folded into running maxima a few per step,
@@ -379,9 +387,15 @@ __device__ __forceinline__ void frag_exp_store_max(const uint32_t (&sv)[64], uin
     for (int e = 0; e < 2; ++e) {
       const uint64_t x =
           fma2(pack2(__uint_as_float(sv[4 * k + 2 * e]), __uint_as_float(sv[4 * k + 2 * e + 1])), c2, nm2[e]);
-      float x0, x1;
-      unpack2(x, x0, x1);
-      const float p0 = fast_exp2(x0), p1 = fast_exp2(x1);
+      float p0, p1;
+      if (frag_exp_on_fma(k, e)) {
+        unpack2(exp2_poly_pair(x), p0, p1);
+      } else {
+        float x0, x1;
+        unpack2(x, x0, x1);
+        p0 = fast_exp2(x0);
+        p1 = fast_exp2(x1);
+      }
       lacc[e][k & 1] = add2(lacc[e][k & 1], pack2(p0, p1));
       w[2 * k + e] = pack_bf16(p0, p1);
     }
