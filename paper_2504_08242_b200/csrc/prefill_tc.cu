@@ -1,23 +1,19 @@
 // Chunked-prefill attention on the 5th-generation tensor cores (paper Sec. IV-A, Fig. 5(b)):
-// chunk rows at positions pos..pos+n-1 attend causally to cache rows 0..pos+i.
+// chunk rows at positions pos..pos+n-1 attend causally to cache rows 0..pos+i.  head_dim 128.
 //
-// head_dim 128.  One CTA owns NQ query tiles of 128 rows of one (sequence, query head) and
-// walks the KV cache in tiles of 128 keys:
-//   loader warp  : TMA (tiled, 128-byte swizzle) Q once, then K/V tiles into 2-stage rings
-//   MMA warp     : one thread issues tcgen05.mma  S = Q K^T  and  O += P V, accumulators in TMEM
-//   softmax WGs  : one warpgroup per query tile, one thread per row, two passes over the S row in
-//                  TMEM (tcgen05.ld): first the masked row maximum (independent 3-input max chains),
-//                  then P = exp2(...) with fp32-pair arithmetic written back in place as bf16
-//                  (aliasing S; 32 columns in flight while 32 are processed); running sum in fp32;
-//                  lazy rescale of O only when the row maximum grew by > 2^8
-// TMEM (512 columns): NQ = 2: S_A | S_B | O_A | O_B (128 each);  NQ = 1: S0 | S1 | O.
-// Key-split mode (SPLIT, the NQ = 2 resources on ONE query tile) for grids that cannot fill the SMs:
-// the two warpgroups run two independent online-softmax streams over the even and the odd KV tiles
-// of the same query tile (one exp2 stream per warpgroup doubles the special-function throughput on
-// the critical path); the streams' (O, m, l) are merged at the end, each warpgroup reading both
-// accumulators from TMEM and writing half of the output columns.
-// All mbarrier waits are bounded; on expiry the CTA sets the status word, drains its own
-// copies and MMAs, frees TMEM and returns.
+// Two kernels, chosen by the size of the grid (see launch_tc):
+//  - prefill_tc_kernel (this file): one CTA owns TWO query tiles of 128 rows of one (sequence, query head) and walks
+//    the KV cache in tiles of 128 keys, every K/V tile serving both query tiles:
+//      loader warp : TMA (tiled, 128-byte swizzle) Q once, then K/V tiles into 2-stage rings
+//      MMA warp    : one thread issues tcgen05.mma  S = Q K^T  and  O += P V, accumulators in TMEM
+//      softmax WGs : one warpgroup per query tile, one thread per row holding the row's 128 scores in registers:
+//                    row maximum, P = exp2(...) with fp32-pair arithmetic written back over S as bf16 and released
+//                    to the MMA issuer in two parts; lazy rescale of O only when the maximum grew by > 2^8
+//    TMEM (512 columns): S_A | S_B | O_A | O_B (128 each).  For grids that cannot fill the SMs a cluster of 4 CTAs
+//    shares the pair of query tiles and splits the KV walk (template parameter CL).
+//  - prefill_frag_kernel (prefill_tc_frag.cuh): one query tile per CTA, both warpgroups on it.
+// All mbarrier waits are bounded; on expiry the CTA sets the status word, drains its own copies and MMAs, frees
+// TMEM and returns.
 #include "host_checks.h"
 #include <atomic>
 
@@ -38,7 +34,7 @@ constexpr int TC_CLUSTER_MIN_TILES = 18;     // shortest KV walk (in tiles) that
 struct TcParams {
   int q_heads, group, q_len, pos, batch;
   int prefix_len;  // rows of a shared prefix cache attended before the sequence's own cache (0: none)
-  int q_blocks;  // ceil(q_len / (128 * NQ))
+  int q_blocks;  // query tiles (fragment form) or pairs of query tiles per (sequence, head)
   float scale_log2;
   float* out;
   float* lse;
@@ -55,24 +51,21 @@ struct TcParams {
 constexpr int TC_PART_FLOATS = 2 * TC_BM * TC_D;  // one CTA's partial accumulators (both query tiles)
 constexpr int TC_ML_FLOATS = 2 * TC_BM * 2;       // one CTA's (m, l) pairs
 
-template <int NQ, bool SPLIT>
+constexpr int TC_NQ = 2;  // query tiles per CTA
 struct TcCfg {
-  static_assert(!SPLIT || NQ == 2, "key-split mode uses the two-tile resources");
-  static constexpr int KV_STAGES = SPLIT ? 3 : 2;
-  static constexpr int Q_TILES = SPLIT ? 1 : NQ;
-  static constexpr int SOFTMAX_WARPS = 4 * NQ;
+  static constexpr int KV_STAGES = 2;
+  static constexpr int SOFTMAX_WARPS = 4 * TC_NQ;
   static constexpr int LOADER_WARP = SOFTMAX_WARPS;
   static constexpr int MMA_WARP = SOFTMAX_WARPS + 1;
-  // The two-warpgroup forms run three full warpgroups (the third: loader, MMA issuer, two idle warps) so that the
-  // register file can be re-divided: a softmax thread holds a whole score row (REGS_SOFTMAX), the third warpgroup
-  // gives its share back (REGS_OTHER); 2 x 128 x 208 + 128 x 88 = 384 x 168, the registers the CTA starts with.
-  static constexpr int THREADS = NQ == 2 ? 384 : 32 * (SOFTMAX_WARPS + 2);
+  // Three full warpgroups (the third: loader, MMA issuer, two idle warps) so that the register file can be
+  // re-divided: a softmax thread holds a whole score row (REGS_SOFTMAX), the third warpgroup gives its share back
+  // (REGS_OTHER); 2 x 128 x 208 + 128 x 88 = 384 x 168, the registers the CTA starts with.
+  static constexpr int THREADS = 384;
   static constexpr int REGS_SOFTMAX = 208, REGS_OTHER = 88;
-  static constexpr int S_BUFS = NQ == 1 ? 2 : 1;  // S buffers per query tile
   static constexpr int O_COL0 = 256;
   // shared memory: [Q tiles][K ring][V ring][barriers]
   static constexpr int SMEM_Q = 0;
-  static constexpr int SMEM_K = Q_TILES * TC_TILE_BYTES;
+  static constexpr int SMEM_K = TC_NQ * TC_TILE_BYTES;
   static constexpr int SMEM_V = SMEM_K + KV_STAGES * TC_TILE_BYTES;
   static constexpr int SMEM_BAR = SMEM_V + KV_STAGES * TC_TILE_BYTES;
   static constexpr int SMEM_BYTES = SMEM_BAR + 256 + 1024;  // + slack for 1024-byte alignment
@@ -82,32 +75,32 @@ struct TcCfg {
 // barrier indices (8 bytes each) inside the barrier block
 enum {
   BAR_Q_FULL = 0,    // [2]
-  BAR_K_FULL = 2,    // [3]
-  BAR_K_EMPTY = 5,   // [3]
-  BAR_V_FULL = 8,    // [3]
-  BAR_V_EMPTY = 11,  // [3]
-  BAR_S_FULL = 14,   // [2 tiles][2 bufs]
-  BAR_P_FULL = 18,   // [2]
-  BAR_O_READY = 20,  // [2]
-  BAR_DRAIN = 22,
-  BAR_STORED = 23,   // the loader's cache stores have read their K/V slots
-  BAR_P_EARLY = 24,  // [2] the first 96 columns of P are in TMEM
-  BAR_COUNT = 26
+  BAR_K_FULL = 2,    // [2]
+  BAR_K_EMPTY = 4,   // [2]
+  BAR_V_FULL = 6,    // [2]
+  BAR_V_EMPTY = 8,   // [2]
+  BAR_S_FULL = 10,   // [2] one per query tile
+  BAR_P_FULL = 12,   // [2]
+  BAR_O_READY = 14,  // [2]
+  BAR_P_EARLY = 16,  // [2] the first 96 columns of P are in TMEM
+  BAR_DRAIN = 18,
+  BAR_COUNT = 19
 };
 
 constexpr int TC_BOX_FLOATS = TC_BM * 32;  // 16 KB
+constexpr int NQ = TC_NQ;
 
 // CL > 1: a thread-block cluster of CL CTAs shares one pair of query tiles; CTA r takes the KV tiles
 // r, r + CL, r + 2 CL, ... and the partial (O, m, l) are exchanged through global scratch (L2) around one
 // cluster barrier: distributed shared memory moved them at about 20 GB/s per SM when measured, L2 is
 // several times faster.  CTA r then finishes the output columns [128 r / CL, 128 (r + 1) / CL).
-template <int NQ, bool SPLIT, int CL>
-__global__ void __launch_bounds__(TcCfg<NQ, SPLIT>::THREADS, 1)
+template <int CL>
+__global__ void __launch_bounds__(TcCfg::THREADS, 1)
 prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                   const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_pk,
                   const __grid_constant__ CUtensorMap tm_pv, const __grid_constant__ CUtensorMap tm_o,
                   const __grid_constant__ CUtensorMap tm_ck, const __grid_constant__ CUtensorMap tm_cv, TcParams p) {
-  using Cfg = TcCfg<NQ, SPLIT>;
+  using Cfg = TcCfg;
   constexpr int KV_STAGES = Cfg::KV_STAGES;
   extern __shared__ unsigned char smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -118,9 +111,8 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem_gen + Cfg::SMEM_BAR + 8 * BAR_COUNT + 8);
   auto bar = [&](int i) { return sBar + 8u * i; };
 
-  static_assert(CL == 1 || (NQ == 2 && !SPLIT), "the cluster mode is built on the two-tile kernel");
-  // a stream of a partial mode can meet rows that see none of a tile, and ends with unnormalised partials
-  constexpr bool PARTIAL = SPLIT || CL > 1;
+  // a CTA of a cluster can meet rows that see none of a tile, and ends with unnormalised partials
+  constexpr bool PARTIAL = CL > 1;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int crank = CL > 1 ? static_cast<int>(cluster_ctarank()) : 0;
 
@@ -133,32 +125,23 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
   // KV tiles 0..Tp-1 come from the shared prefix (every row sees them, no causal limit), the rest from
   // the sequence's own cache
   const int Tp = (p.prefix_len + TC_BN - 1) / TC_BN;
-  // T[x]: KV tiles of softmax stream x; Tall: KV tiles the CTA loads (its load sequence 0..Tall-1).
-  // Stream x of the key-split mode takes the sequence numbers 2 i + x of its (single) query tile; CTA r
-  // of a cluster loads KV tile r + CL n as its n-th.
+  // T[x]: KV tiles of query tile x; Tall: KV tiles the CTA loads (its load sequence 0..Tall-1).  CTA r of a
+  // cluster loads KV tile r + CL n as its n-th.
   int T[2] = {0, 0};
   int Tg[2] = {0, 0};  // cluster mode: tiles of the query tile over the whole cluster
-  int Tall;
-  if constexpr (SPLIT) {
-    Tall = Tp + (p.pos + min(p.q_len, (qblk + 1) * TC_BM) + TC_BN - 1) / TC_BN;
-    T[0] = (Tall + 1) >> 1;
-    T[1] = Tall >> 1;
-  } else {
+#pragma unroll
+  for (int x = 0; x < NQ; ++x) {
+    const int r0 = (qblk * NQ + x) * TC_BM;
+    if (r0 < p.q_len) T[x] = Tp + (p.pos + min(p.q_len, r0 + TC_BM) + TC_BN - 1) / TC_BN;
+  }
+  if constexpr (CL > 1) {
 #pragma unroll
     for (int x = 0; x < NQ; ++x) {
-      const int r0 = (qblk * NQ + x) * TC_BM;
-      if (r0 < p.q_len) T[x] = Tp + (p.pos + min(p.q_len, r0 + TC_BM) + TC_BN - 1) / TC_BN;
+      Tg[x] = T[x];
+      T[x] = T[x] > crank ? (T[x] - crank + CL - 1) / CL : 0;
     }
-    if constexpr (CL > 1) {
-#pragma unroll
-      for (int x = 0; x < NQ; ++x) {
-        Tg[x] = T[x];
-        T[x] = T[x] > crank ? (T[x] - crank + CL - 1) / CL : 0;
-      }
-    }
-    Tall = NQ == 2 ? max(T[0], T[1]) : T[0];
   }
-  auto seq_of = [](int x, int i) { return SPLIT ? 2 * i + x : i; };  // load sequence number of stream x's i-th step
+  const int Tall = max(T[0], T[1]);
   auto tile_of_seq = [&](int n) { return CL > 1 ? crank + CL * n : n; };  // KV tile of a sequence number
 
   // ---- set-up
@@ -195,12 +178,12 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
 
   if (warp == Cfg::LOADER_WARP) {
     // =============================================================== loader
-    if constexpr (NQ == 2) reg_dec<Cfg::REGS_OTHER>();
+    reg_dec<Cfg::REGS_OTHER>();
     if (lane == 0) {
 #pragma unroll
-      for (int x = 0; x < Cfg::Q_TILES; ++x) {
+      for (int x = 0; x < NQ; ++x) {
         if (T[x] == 0) continue;
-        const int r0 = (SPLIT ? qblk : qblk * NQ + x) * TC_BM;
+        const int r0 = (qblk * NQ + x) * TC_BM;
         mbar_expect_tx(bar(BAR_Q_FULL + x), TC_TILE_BYTES);
         tma_load_4d(sQ + x * TC_TILE_BYTES, &tm_q, bar(BAR_Q_FULL + x), 0, h, r0, b);
         tma_load_4d(sQ + x * TC_TILE_BYTES + TC_PANEL_BYTES, &tm_q, bar(BAR_Q_FULL + x), 64, h, r0, b);
@@ -210,7 +193,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
       // Fused KVCache write: the chunk's own K/V tiles are loaded for the attention anyway; the tiles that hold
       // the query rows of this CTA (of this cluster: the CTA that loads them) go from their slots to the cache with
       // tiled stores, as soon as they have landed.  A slot is refilled only after its store has read it.
-      constexpr int QT = SPLIT ? 1 : NQ;  // query tiles of the chunk per CTA (cluster)
+      constexpr int QT = NQ;  // query tiles of the chunk per CTA (cluster)
       const bool writer = p.fused_write != 0 && h % p.group == 0;
       auto store_own_tile = [&](int j) {  // j: load sequence number
         const int t = tile_of_seq(j) - Tp;  // tile of the chunk
@@ -251,7 +234,6 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         issued = 2 * j + 2;
       }
       for (int j = max(0, Tall - KV_STAGES); j < Tall && ok; ++j) store_own_tile(j);
-      mbar_arrive(bar(BAR_STORED));  // the slots may be reused as scratch (key-split merge)
       if (*abort_flag) {
         // wait (bounded) until every copy this thread started has landed before shared memory is released
         int dummy = 0;
@@ -261,26 +243,26 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
           mbar_wait(bar(BAR_K_FULL + j % KV_STAGES), (j / KV_STAGES) & 1, none, nullptr);
         for (int j = max(0, nv - KV_STAGES); j < nv; ++j)
           mbar_wait(bar(BAR_V_FULL + j % KV_STAGES), (j / KV_STAGES) & 1, none, nullptr);
-        for (int x = 0; x < Cfg::Q_TILES; ++x)
+        for (int x = 0; x < NQ; ++x)
           if (T[x] > 0) mbar_wait(bar(BAR_Q_FULL + x), 0, none, nullptr);
       }
     }
     __syncwarp();
   } else if (warp == Cfg::MMA_WARP) {
     // =============================================================== MMA issuer
-    if constexpr (NQ == 2) reg_dec<Cfg::REGS_OTHER>();
+    reg_dec<Cfg::REGS_OTHER>();
     if (lane == 0) {
       constexpr uint32_t idesc_qk = tc_idesc_bf16(TC_BM, TC_BN, false, false);
       constexpr uint32_t idesc_pv = tc_idesc_bf16(TC_BM, TC_D, false, true);
-      auto s_col = [&](int x, int buf) { return tmem + (NQ == 2 ? x * 128 : buf * 128); };
+      auto s_col = [&](int x) { return tmem + x * 128; };
       auto o_col = [&](int x) { return tmem + Cfg::O_COL0 + x * 128; };
       // The issue loops are kept to an integer addition or two per MMA (descriptor halves, see tc_desc_lo): this
       // thread shares its scheduler with two softmax warps, and a longer chain of address arithmetic per MMA
       // made the issue, not the tensor pipe, the limit.
-      auto issue_qk = [&](int x, int g, int buf) {  // S(x) = Q(x) K^T, K of load sequence number g
-        const uint32_t q_lo = tc_desc_lo(sQ + (SPLIT ? 0 : x) * TC_TILE_BYTES, 16);
+      auto issue_qk = [&](int x, int g) {  // S(x) = Q(x) K^T, K of load sequence number g
+        const uint32_t q_lo = tc_desc_lo(sQ + x * TC_TILE_BYTES, 16);
         const uint32_t k_lo = tc_desc_lo(sK + (g % KV_STAGES) * TC_TILE_BYTES, 16);
-        const uint32_t d = s_col(x, buf);
+        const uint32_t d = s_col(x);
 #pragma unroll
         for (int ks = 0; ks < TC_D / 16; ++ks) {
           const uint32_t off = ((ks >> 2) * TC_PANEL_BYTES + (ks & 3) * 32) >> 4;
@@ -288,15 +270,14 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         }
       };
       // O(x) (+)= P(x) V over the keys [16 ks0, 16 ks1) of the tile, V of load sequence number g
-      auto issue_pv = [&](int x, int g, int buf, bool first, int ks0, int ks1) {
+      auto issue_pv = [&](int x, int g, bool first, int ks0, int ks1) {
         const uint32_t v_lo = tc_desc_lo(sV + (g % KV_STAGES) * TC_TILE_BYTES, TC_PANEL_BYTES);
-        const uint32_t d = o_col(x), a = s_col(x, buf);
+        const uint32_t d = o_col(x), a = s_col(x);
 #pragma unroll
         for (int ks = ks0; ks < ks1; ++ks)
           tc_mma_ts_lo(d, a + ks * 8, v_lo + ks * (2048 >> 4), idesc_pv, (!first || ks > 0));
       };
-      auto last_user = [&](int g) {  // the last stream (in issue order) that uses the tile of sequence number g
-        if (SPLIT) return g & 1;
+      auto last_user = [&](int g) {  // the last query tile (in issue order) that uses the tile of sequence number g
         int r = -1;
 #pragma unroll
         for (int x = 0; x < NQ; ++x)
@@ -323,44 +304,34 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
 #pragma unroll
       for (int x = 0; x < NQ; ++x) {
         if (T[x] == 0 || !ok) continue;
-        if (!SPLIT || x == 0) ok = ok && mbar_wait(bar(BAR_Q_FULL + x), 0, abort_flag, p.status);
-        const int g = seq_of(x, 0);
-        need_k(g);
+        ok = ok && mbar_wait(bar(BAR_Q_FULL + x), 0, abort_flag, p.status);
+        need_k(0);
         if (!ok) break;
-        issue_qk(x, g, 0);
-        tc_commit(bar(BAR_S_FULL + 2 * x + 0));
-        if (x == last_user(g)) tc_commit(bar(BAR_K_EMPTY + g % KV_STAGES));
+        issue_qk(x, 0);
+        tc_commit(bar(BAR_S_FULL + x));
+        if (x == last_user(0)) tc_commit(bar(BAR_K_EMPTY + 0));
       }
-      const int Tsteps = NQ == 2 ? max(T[0], T[1]) : T[0];
-      for (int j = 0; j < Tsteps && ok; ++j) {
+      for (int j = 0; j < Tall && ok; ++j) {
 #pragma unroll
         for (int x = 0; x < NQ; ++x) {
           if (j >= T[x] || !ok) continue;
-          const int buf = NQ == 1 ? (j & 1) : 0;
-          const int g = seq_of(x, j), gn = seq_of(x, j + 1);  // load sequence numbers
-          if (NQ == 1 && j + 1 < T[x]) {  // next S into the other buffer while the softmax works on this one
-            need_k(gn);
-            if (!ok) break;
-            issue_qk(x, gn, (j + 1) & 1);
-            tc_commit(bar(BAR_S_FULL + 2 * x + ((j + 1) & 1)));
-            tc_commit(bar(BAR_K_EMPTY + gn % KV_STAGES));
-          }
+          const int g = j, gn = j + 1;  // load sequence numbers
           need_v(g);
           ok = ok && mbar_wait(bar(BAR_P_EARLY + x), j & 1, abort_flag, p.status);
           if (!ok) break;
           tc_fence_after();
-          issue_pv(x, g, buf, j == 0, 0, 6);  // the first 96 keys while the softmax finishes the last 32
+          issue_pv(x, g, j == 0, 0, 6);  // the first 96 keys while the softmax finishes the last 32
           ok = ok && mbar_wait(bar(BAR_P_FULL + x), j & 1, abort_flag, p.status);
           if (!ok) break;
           tc_fence_after();
-          issue_pv(x, g, buf, j == 0, 6, 8);
+          issue_pv(x, g, j == 0, 6, 8);
           tc_commit(bar(BAR_O_READY + x));
           if (x == last_user(g)) tc_commit(bar(BAR_V_EMPTY + g % KV_STAGES));
-          if (NQ == 2 && j + 1 < T[x]) {
+          if (j + 1 < T[x]) {
             need_k(gn);
             if (!ok) break;
-            issue_qk(x, gn, 0);
-            tc_commit(bar(BAR_S_FULL + 2 * x));
+            issue_qk(x, gn);
+            tc_commit(bar(BAR_S_FULL + x));
             if (x == last_user(gn)) tc_commit(bar(BAR_K_EMPTY + gn % KV_STAGES));
           }
         }
@@ -374,10 +345,10 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     __syncwarp();
   } else if (warp < Cfg::SOFTMAX_WARPS) {
     // =============================================================== softmax warpgroups
-    if constexpr (NQ == 2) reg_inc<Cfg::REGS_SOFTMAX>();
-    const int x = warp >> 2;                      // query tile (key-split mode: stream) of this warpgroup
+    reg_inc<Cfg::REGS_SOFTMAX>();
+    const int x = warp >> 2;                      // query tile of this warpgroup
     const int row_in_tile = (warp & 3) * 32 + lane;
-    const int row = (SPLIT ? qblk : qblk * NQ + x) * TC_BM + row_in_tile;  // row inside the chunk
+    const int row = (qblk * NQ + x) * TC_BM + row_in_tile;  // row inside the chunk
     const bool row_valid = row < p.q_len;
     const int lim = p.pos + min(row, p.q_len - 1) + 1;      // keys j < lim are visible
     const uint32_t lane_base = static_cast<uint32_t>((warp & 3) * 32) << 16;
@@ -387,14 +358,12 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     bool ok = true;
     const int Tx = T[x];
     for (int j = 0; j < Tx && ok; ++j) {
-      const int buf = NQ == 1 ? (j & 1) : 0;
-      const uint32_t tS = tmem + lane_base + (NQ == 2 ? x * 128 : buf * 128);
-      const uint32_t s_parity = NQ == 1 ? ((j >> 1) & 1) : (j & 1);
-      ok = mbar_wait(bar(BAR_S_FULL + 2 * x + buf), s_parity, abort_flag, p.status);
+      const uint32_t tS = tmem + lane_base + x * 128;
+      ok = mbar_wait(bar(BAR_S_FULL + x), j & 1, abort_flag, p.status);
       if (!ok) break;
       tc_fence_after();
       // columns >= nvalid are masked: the end of the prefix in its last tile, the causal limit afterwards
-      const int g = tile_of_seq(seq_of(x, j));
+      const int g = tile_of_seq(j);
       const int nvalid = g < Tp ? p.prefix_len - g * TC_BN : lim - (g - Tp) * TC_BN;
       // warp-uniform flag, so the warp stays converged for the collective tcgen05 operations
       const bool masked = __any_sync(0xffffffffu, nvalid < TC_BN);
@@ -417,63 +386,6 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
       if (Tx > 0) ok = mbar_wait(bar(BAR_O_READY + x), (Tx - 1) & 1, abort_flag, p.status) && ok;
       part_m = m_ref;
       part_l = l;
-    } else if constexpr (SPLIT) {
-      // Merge of the two streams.  Every softmax thread reaches the named barriers below, even one that gave
-      // up on a wait (it only skips its global stores).  (m, l) of a row cross through shared memory; the
-      // accumulators are read straight from TMEM: this warpgroup combines columns [64 x, 64 x + 64) of both.
-      // The K slot of a stream's last tile is free once its S has been seen (no later tile maps to it), so it
-      // carries that stream's (m, l); a stream without tiles owns slot 1, which was never filled.
-      auto ml_of = [&](int y) {
-        return reinterpret_cast<float2*>(smem_gen + Cfg::SMEM_K + (seq_of(y, max(T[y] - 1, 0)) % KV_STAGES) * TC_TILE_BYTES);
-      };
-      ok = mbar_wait(bar(BAR_STORED), 0, abort_flag, p.status) && ok;  // no cache store still reads the slots
-      ml_of(x)[row_in_tile] = make_float2(m_ref, l);
-      if (Tx > 0) ok = mbar_wait(bar(BAR_O_READY + x), (Tx - 1) & 1, abort_flag, p.status) && ok;
-      tc_fence_before();
-      asm volatile("bar.sync 3, 256;\n" ::: "memory");
-      tc_fence_after();
-      const float2 oth = ml_of(1 - x)[row_in_tile];
-      // a stream whose tiles were all hidden from this row has l = 0 and takes no part
-      const float m_own = l > 0.f ? m_ref : -INFINITY, m_oth = oth.y > 0.f ? oth.x : -INFINITY;
-      const float m = fmaxf(m_own, m_oth);
-      const float w_own = l > 0.f ? fast_exp2(m_own - m) : 0.f, w_oth = oth.y > 0.f ? fast_exp2(m_oth - m) : 0.f;
-      const float lsum = l * w_own + oth.y * w_oth;
-      const float inv = 1.f / lsum;
-      const float a_own = w_own * inv, a_oth = w_oth * inv;
-      const bool has_own = Tx > 0, has_oth = T[1 - x] > 0;  // a stream without tiles never wrote its accumulator
-      const uint32_t tOwn = tmem + lane_base + Cfg::O_COL0 + x * 128 + x * 64;
-      const uint32_t tOth = tmem + lane_base + Cfg::O_COL0 + (1 - x) * 128 + x * 64;
-      // staging: the Q buffer for stream 0, the first V slot for stream 1 (every MMA and copy is complete)
-      float* stage = reinterpret_cast<float*>(smem_gen + (x == 0 ? Cfg::SMEM_Q : Cfg::SMEM_V));
-      const int tid_t = threadIdx.x & 127;
-      const int tile_row0 = qblk * TC_BM;
-      // two boxes of 128 rows x 32 columns; each goes out as a tiled store as soon as it is staged, so the second
-      // box is staged while the first is being read; rows at or beyond q_len are clipped by the tensor map
-#pragma unroll
-      for (int q2 = 0; q2 < 2; ++q2) {
-        uint32_t o[32], o2[32];
-        if (has_own) tmem_ld32(tOwn + q2 * 32, o);
-        if (has_oth) tmem_ld32(tOth + q2 * 32, o2);
-        tc_wait_ld();
-        float v[32];
-#pragma unroll
-        for (int i = 0; i < 32; ++i) {
-          v[i] = has_own ? __uint_as_float(o[i]) * a_own : 0.f;
-          if (has_oth) v[i] = fmaf(__uint_as_float(o2[i]), a_oth, v[i]);
-        }
-        stage_box_row(stage + q2 * TC_BOX_FLOATS, row_in_tile, v);
-        fence_proxy_async();
-        asm volatile("bar.sync %0, 128;\n" ::"r"(1 + x) : "memory");
-        if (tid_t == 0 && ok) {
-          const uint32_t src = smem_base + (x == 0 ? Cfg::SMEM_Q : Cfg::SMEM_V);
-          tma_store_4d(&tm_o, src + q2 * TC_BOX_FLOATS * 4, x * 64 + q2 * 32, h, tile_row0, b);
-          tma_store_commit();
-        }
-      }
-      if (tid_t == 0) tma_store_wait_read();  // shared memory is released at the end of the kernel; the writes complete with the grid
-      if (x == 0 && ok && p.lse && row_valid)
-        p.lse[(static_cast<int64_t>(b) * p.q_heads + h) * p.q_len + row] =
-            (m + log2f(lsum)) * 0.69314718055994530942f;
     } else if (Tx > 0) {  // warpgroup-uniform: every thread of the tile reaches the named barriers below, even
                           // one that gave up on a wait (it only skips its global stores)
       ok = ok && mbar_wait(bar(BAR_O_READY + x), (Tx - 1) & 1, abort_flag, p.status);
@@ -515,7 +427,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     }
   }
 
-  else if constexpr (NQ == 2) {
+  else {
     reg_dec<Cfg::REGS_OTHER>();  // the idle warps of the third warpgroup: the re-division is a warpgroup's decision
   }
 
@@ -670,23 +582,23 @@ static cudaError_t launch_frag(int64_t ctas, cudaStream_t st, const CUtensorMap&
                             FragCfg::SMEM_BYTES, st, 1u, tq, tk, tv, tpk, tpv, tck, tcv, p);
 }
 
-template <int NQ, bool SPLIT, int CL>
+template <int CL>
 static cudaError_t launch_variant(int64_t ctas, cudaStream_t st, const CUtensorMap& tq, const CUtensorMap& tk,
                                   const CUtensorMap& tv, const CUtensorMap& tpk, const CUtensorMap& tpv,
                                   const CUtensorMap& to, const CUtensorMap& tck, const CUtensorMap& tcv,
                                   const TcParams& p) {
-  using Cfg = TcCfg<NQ, SPLIT>;
+  using Cfg = TcCfg;
   static PerDeviceOnce done;
   if (!done.done()) {
     cudaError_t e =
-        cudaFuncSetAttribute(prefill_tc_kernel<NQ, SPLIT, CL>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM_BYTES);
+        cudaFuncSetAttribute(prefill_tc_kernel<CL>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM_BYTES);
     if (e == cudaSuccess)
-      e = cudaFuncSetAttribute(prefill_tc_kernel<NQ, SPLIT, CL>, cudaFuncAttributePreferredSharedMemoryCarveout,
+      e = cudaFuncSetAttribute(prefill_tc_kernel<CL>, cudaFuncAttributePreferredSharedMemoryCarveout,
                                cudaSharedmemCarveoutMaxShared);
     if (e != cudaSuccess) return e;
     done.set();
   }
-  return launch_pdl_cluster(prefill_tc_kernel<NQ, SPLIT, CL>, dim3(static_cast<unsigned>(ctas * CL)),
+  return launch_pdl_cluster(prefill_tc_kernel<CL>, dim3(static_cast<unsigned>(ctas * CL)),
                             dim3(Cfg::THREADS), Cfg::SMEM_BYTES, st, static_cast<unsigned>(CL), tq, tk, tv, tpk, tpv, to, tck,
                             tcv, p);
 }
@@ -699,9 +611,9 @@ static int max_resident_clusters() {
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 0;
   const int cached = cache[dev].load(std::memory_order_acquire);
   if (cached > 0) return cached - 1;
-  using Cfg = TcCfg<2, false>;
+  using Cfg = TcCfg;
   int n = 0;
-  if (cudaFuncSetAttribute(prefill_tc_kernel<2, false, CL>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+  if (cudaFuncSetAttribute(prefill_tc_kernel<CL>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            Cfg::SMEM_BYTES) == cudaSuccess) {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(CL * 64);
@@ -715,7 +627,7 @@ static int max_resident_clusters() {
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     int got = 0;
-    if (cudaOccupancyMaxActiveClusters(&got, prefill_tc_kernel<2, false, CL>, &cfg) == cudaSuccess) n = got;
+    if (cudaOccupancyMaxActiveClusters(&got, prefill_tc_kernel<CL>, &cfg) == cudaSuccess) n = got;
     else (void)cudaGetLastError();
   } else {
     (void)cudaGetLastError();
@@ -801,14 +713,11 @@ static cudaError_t launch_tc(const bf16* q, const CacheView& c, const CacheView*
   p.out = out;
   p.lse = lse;
   p.status = status;
-  // Two query tiles per CTA when that still fills the machine.  A grid that leaves SMs idle is latency-bound
-  // on the walk over the KV tiles.  With query tiles in pairs and a long walk, a cluster of 4 CTAs shares it:
-  // the exchange of the partials costs about 10 us, the key-split streams of the one-tile form advance by about
-  // one tile per us and the cluster by four, so the cluster pays from about 18 tiles on (measured, chunk 256 x 32
-  // heads, one eager launch: 16 tiles 29.7 us either way, 20 tiles 31.6 against 33.8, 24 tiles 33.7 against 37.8,
-  // 66 tiles 61 against 84; and only while all clusters are resident at
-  // once).  Otherwise one tile per CTA, with both warpgroups on it (key-split streams) while a single wave
-  // holds every CTA, else with one.
+  // Two query tiles per CTA when that still fills the machine (every K/V tile then serves two query tiles).  A
+  // grid that leaves SMs idle is latency-bound on the walk over the KV tiles: with few pairs of query tiles and a
+  // long walk, a cluster of 4 CTAs shares a pair and splits the walk; the exchange of the partials costs about
+  // 10 us, so the cluster pays from about 18 KV tiles on (measured on chunk 256 x 32 heads), and only while all
+  // clusters are resident at once.  Otherwise one query tile per CTA (fragment form).
   const int64_t ctas2 = static_cast<int64_t>((q_len + 255) / 256) * c.batch * q_heads;
   const int64_t ctas1 = static_cast<int64_t>((q_len + 127) / 128) * c.batch * q_heads;
   const int kv_tiles = (prefix_len + TC_BN - 1) / TC_BN + (pos + q_len + TC_BN - 1) / TC_BN;
@@ -826,10 +735,10 @@ static cudaError_t launch_tc(const bf16* q, const CacheView& c, const CacheView*
   cudaError_t e;
   if (ctas2 >= li.sm_count) {
     p.q_blocks = (q_len + 255) / 256;
-    e = launch_variant<2, false, 1>(ctas2, st, tq, tk, tv, tpk, tpv, to, tck, tcv, p);
+    e = launch_variant<1>(ctas2, st, tq, tk, tv, tpk, tpv, to, tck, tcv, p);
   } else if (cl == 4) {
     p.q_blocks = (q_len + 255) / 256;
-    e = launch_variant<2, false, 4>(ctas2, st, tq, tk, tv, tpk, tpv, to, tck, tcv, p);
+    e = launch_variant<4>(ctas2, st, tq, tk, tv, tpk, tpv, to, tck, tcv, p);
   } else {
     p.q_blocks = (q_len + 127) / 128;
     e = launch_frag(ctas1, st, tq, tk, tv, tpk, tpv, tck, tcv, p);

@@ -311,57 +311,13 @@ __device__ __forceinline__ bool frag_decide(const float (&mxs)[2], float (&m_ref
   return true;
 }
 
-// P = exp2(s c - m_ref) as bf16 pairs over the first 64 columns of the tile's S buffer, row sums into l; mid() runs
-// after the first half (the caller's work on the next tile goes there).  Returns with the stores issued, not waited.
-template <class Mid>
-__device__ __forceinline__ void frag_exp_store(const uint32_t (&sv)[64], uint32_t tS, float c, const float (&m_ref)[2],
-                                               float (&l)[2], Mid&& mid) {
-  uint64_t nm2[2];
-#pragma unroll
-  for (int e = 0; e < 2; ++e) {
-    const float nm = m_ref[e] == -INFINITY ? 0.f : -m_ref[e];
-    nm2[e] = pack2(nm, nm);
-  }
-  const uint64_t c2 = pack2(c, c);
-  uint64_t lacc[2][2];
-#pragma unroll
-  for (int e = 0; e < 2; ++e) lacc[e][0] = lacc[e][1] = pack2(0.f, 0.f);
-  uint32_t w[32];  // P: w[2k + e] = keys 8k + col0 + {0, 1} of row e
-#pragma unroll
-  for (int k = 0; k < 16; ++k) {
-#pragma unroll
-    for (int e = 0; e < 2; ++e) {
-      const uint64_t x =
-          fma2(pack2(__uint_as_float(sv[4 * k + 2 * e]), __uint_as_float(sv[4 * k + 2 * e + 1])), c2, nm2[e]);
-      float x0, x1;
-      unpack2(x, x0, x1);
-      const float p0 = fast_exp2(x0), p1 = fast_exp2(x1);
-      lacc[e][k & 1] = add2(lacc[e][k & 1], pack2(p0, p1));
-      w[2 * k + e] = pack_bf16(p0, p1);
-    }
-    if (k == 7) {
-      tmem_st_16x128b_x8(tS, &w[0]);
-      mid();
-    }
-  }
-  tmem_st_16x128b_x8(tS + 32, &w[16]);
-#pragma unroll
-  for (int e = 0; e < 2; ++e) {
-    float a0, a1;
-    unpack2(add2(lacc[e][0], lacc[e][1]), a0, a1);
-    l[e] += a0 + a1;
-  }
-}
+// Which of a tile's 32 column pairs per thread (step k, row e) take their exponentials on the FMA pipe: a quarter
+// (more brought nothing: the loop is bound by dependent-issue latency, not by the special-function unit alone).
+__device__ __forceinline__ constexpr bool frag_exp_on_fma(int k, int e) { return e == 1 && (k & 1) != 0; }
 
-// Which of a tile's 32 column pairs per thread (step k, row e) take their exponentials on the FMA pipe.
-#ifndef JUP_EXP_EMU
-#define JUP_EXP_EMU 1
-#endif
-__device__ __forceinline__ constexpr bool frag_exp_on_fma(int k, int e) {
-  return JUP_EXP_EMU == 1 ? (e == 1 && (k & 1)) : JUP_EXP_EMU == 2 ? (e == 1) : JUP_EXP_EMU == 3 ? (e == 1 && (k & 3) == 3) : false;
-}
-
-// The same with the next tile's row maxima worked in: nxt is a fragment load in flight (or stale registers when there
+// P = exp2(s c - m_ref) of a tile held in fragments, as bf16 pairs over the first 64 columns of its S buffer, row
+// sums into l (the stores are issued, not waited for), with the next tile's row maxima worked in: nxt is a fragment
+// load in flight (or stale registers when there
 // is no next tile; the result is then unused).  It is waited for after the fourth of the sixteen steps, masked if
 // need be (mask_next(), warp-uniform and rare), and its 2 x 32 values are folded into running maxima a few per step,
 // so that their arithmetic issues in the gaps of the exponentials instead of after them.  mxs_next: maxima times c.
