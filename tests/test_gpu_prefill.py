@@ -73,20 +73,29 @@ def test_two_query_tiles_per_cta_ragged(ctx):
     check_workload(ctx, w, parts=[515])
 
 
-def test_key_split_streams_one_tile_per_cta(ctx):
-    """Few (sequence, head, 128-row tile) units: both warpgroups of a CTA walk the even and the odd KV
-    tiles of one query tile and merge at the end.  Covers a walk of one tile (the second stream has
-    nothing), rows that see none of a stream's first tile (position not a multiple of 128), a ragged
-    last query tile, and GQA."""
-    w = synth.PrefillWorkload("split_a", 48, 1, 8, 2, 128, 433, 433, 450)
+def test_one_query_tile_per_cta_small_grids(ctx):
+    """Few (sequence, head, 128-row tile) units: one query tile per CTA, both softmax warpgroups on it (16 rows per
+    warp).  Covers walks of one, two and three tiles (the pipeline holds three score buffers; the last three tiles
+    complete the accumulator's own barriers), rows that see none of the last tile (position not a multiple of
+    128), a ragged last query tile, GQA, and LSE."""
+    w = synth.PrefillWorkload("frag_a", 48, 1, 8, 2, 128, 433, 433, 450)
     check_workload(ctx, w, parts=[64, 269, 100], want_lse=True)
-    w = synth.PrefillWorkload("split_b", 49, 2, 4, 4, 128, 1100, 1100, 1100)
+    w = synth.PrefillWorkload("frag_b", 49, 2, 4, 4, 128, 1100, 1100, 1100)
     check_workload(ctx, w, parts=[1, 127, 130, 842], want_lse=True)
 
 
-def test_one_warpgroup_one_tile_variant(ctx):
-    """More 128-row tiles than SMs but too few 256-row pairs to fill them: one query tile per CTA with a
-    single softmax warpgroup and a double-buffered S."""
+@pytest.mark.parametrize("tiles", [1, 2, 3, 4, 5, 7])
+def test_one_query_tile_per_cta_walk_lengths(ctx, tiles):
+    """Every short walk length of the three-buffer pipeline, one call on a cold cache (the unfused call must leave the
+    cache untouched: check_workload compares it bit by bit afterwards)."""
+    S = tiles * 128 - 37
+    w = synth.PrefillWorkload(f"frag_walk_{tiles}", 170 + tiles, 1, 2, 1, 128, S, S, S + 5)
+    first = max(S - 100, 1)
+    check_workload(ctx, w, parts=[first, S - first] if S > first else [S], want_lse=True)
+
+
+def test_one_query_tile_per_cta_more_tiles_than_sms(ctx):
+    """More 128-row tiles than SMs but too few 256-row pairs to fill them: the same form over several waves."""
     w = synth.PrefillWorkload("one_tile", 50, 1, 32, 8, 128, 700, 700, 700)
     check_workload(ctx, w, parts=[60, 640])
 

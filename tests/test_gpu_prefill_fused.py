@@ -56,10 +56,10 @@ def test_every_launch_variant(ctx):
     # two query tiles per CTA (grid fills the GPU), GQA, ragged
     w = synth.PrefillWorkload("fused_two_tiles", 161, 2, 32, 8, 128, 800, 800, 832)
     check(ctx, w, [100, 700], launches_per_chunk=1)
-    # one tile, one warpgroup
+    # one query tile per CTA over several waves
     w = synth.PrefillWorkload("fused_one_tile", 162, 1, 32, 8, 128, 700, 700, 700)
     check(ctx, w, [60, 640], launches_per_chunk=1)
-    # key-split streams (K moved by one warpgroup, V by the other)
+    # one query tile per CTA on a small grid (the loader stores the CTA's own K/V tile from its slots)
     w = synth.PrefillWorkload("fused_split", 163, 1, 8, 2, 128, 433, 433, 450)
     check(ctx, w, [64, 269, 100], launches_per_chunk=1)
     # clusters of four CTAs on a long walk: only the first CTA of a cluster writes the cache
