@@ -1,11 +1,14 @@
-// One online-softmax step of the tcgen05 attention kernels: a thread owns one query row (one TMEM lane) and
-// walks the 128 fp32 scores of the current key tile ONCE, in four chunks of 32 columns (tcgen05.ld, the next chunk
-// in flight while the current one is processed): chunk maximum, then P = exp2(s * c - m) with fp32-pair
-// arithmetic, written back in place as bf16 pairs (P column k holds keys 2k and 2k + 1, so the writes stay behind
-// the reads).  The reference maximum m is lazy: it only moves when a chunk's maximum outgrew it by more than 2^8;
-// then the row sum, the P chunks of this tile written so far and -- at the end of the tile -- the accumulator O are
-// scaled by exp2(m_old - m_new).  With well-behaved scores that happens in a row's first chunk and almost never
-// again, so a tile costs one pass over TMEM instead of a maximum pass plus an exponential pass.
+// The online-softmax steps of the tcgen05 attention kernels, three forms of the same arithmetic -- P = exp2(s c - m)
+// with fp32-pair instructions, written back over S in TMEM as bf16 pairs (P column k holds keys 2k and 2k + 1, so the
+// writes stay behind the reads), a lazy reference maximum m that only moves when the tile's maximum outgrew it by more
+// than 2^8 (then the row sum and the accumulator O are scaled by exp2(m_old - m_new); with well-behaved scores that
+// happens in a row's first tile and almost never again):
+//   softmax_tile_step : a thread per row, the row's 128 scores walked once in four chunks of 32 columns with the next
+//                       chunk in flight (about 160 registers; the branch kernel)
+//   softmax_tile_row  : a thread per row holding the whole row (about 200 registers), P released in two parts (the
+//                       two-tile prefill kernel)
+//   frag_*            : 16 rows per warp in the 16x256b fragment layout, in pieces that a kernel interleaves across
+//                       consecutive tiles (the one-tile prefill kernel)
 #pragma once
 #include "tc_common.cuh"
 
