@@ -69,6 +69,26 @@ def test_every_launch_variant(ctx):
     check(ctx, w, [2980, 384], launches_per_chunk=1)
 
 
+def test_random_geometry(ctx):
+    """Seeded random prompts: batch, head counts and group sizes, prompt lengths and ragged chunkings, so that the three
+    tcgen05 forms (two query tiles per CTA, clusters, one query tile per CTA) and their boundaries are all met; both
+    the fused and the two-call form, every output, LSE and the cache compared."""
+    dims = synth.uniform_ints(91, 1, 10 * 6, 0, 1 << 20).reshape(-1, 6)
+    for k, row in enumerate(dims):
+        B = 1 + int(row[0]) % 3
+        Hkv = [1, 2, 8][int(row[1]) % 3]
+        G = [1, 2, 4][int(row[2]) % 3]
+        S = 150 + int(row[3]) % 1300
+        cuts = sorted(set(int(x) % S for x in synth.uniform_ints(int(row[4]), 2, 1 + int(row[5]) % 4, 1, 1 << 20)) - {0})
+        parts = [b - a for a, b in zip([0] + cuts, cuts + [S])]
+        w = synth.PrefillWorkload(f"fused_random_{k}", 700 + k, B, Hkv * G, Hkv, 128, S, S, S + int(row[5]) % 17)
+        check(ctx, w, parts, launches_per_chunk=1)
+        q, kk, v = w.make()
+        out = run_gpu_prefill(ctx, q, kk, v, parts, w.capacity, w.scale, poison=True, fused=False)[0]
+        ref = oracle.full_causal(q, kk, v, w.scale, n_threads=oracle.hardware_threads())
+        assert_close(out, ref, w.name + " (two calls)")
+
+
 def test_strided_cache(ctx):
     """Row stride larger than the head dimension (a cache that interleaves K and V storage)."""
     import torch
