@@ -586,7 +586,7 @@ TC_SOURCES = ["tc_common.cuh", "tc_softmax.cuh", "common.cuh"]
 PREFILL_SOURCES = ["prefill_tc.cu", "prefill_tc_frag.cuh"] + TC_SOURCES
 TRAFFIC_PROFILES = {
     "cfg2": ("prefill_frag_kernel_cfg2.md", PREFILL_SOURCES),
-    # (chunk 128 runs the one-query-tile kernel, of which there is no capture at this size)
+    "cfg3_c128": ("prefill_frag_kernel_cfg3_c128.md", PREFILL_SOURCES),
     "cfg3_c512": ("prefill_tc_kernel_cfg3_c512.md", PREFILL_SOURCES),
     "cfg3_c1024": ("prefill_tc_kernel_cfg3_c512.md", PREFILL_SOURCES),
     "cfg4": ("branch_stream_kernel_cfg4.md", ["branch_stream.cu", "tc_common.cuh", "common.cuh"]),
